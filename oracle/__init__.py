@@ -1,0 +1,17 @@
+"""fp64 CPU oracle for partial causal attention, its merge and the partition planner.
+
+Test infrastructure only: nothing in the GPU library imports this package, and this
+package imports nothing from the GPU library.
+"""
+from .reference import (  # noqa: F401
+    attn_rows,
+    prefill_attn,
+    varlen_attn,
+    merge,
+    plan_partitions,
+    partition_intervals,
+    oracle_threads,
+    SKIP,
+    PARTIAL,
+    FULL,
+)

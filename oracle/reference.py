@@ -1,0 +1,222 @@
+"""Oracle entry points (test infrastructure; see pec_oracle.c for the attention arithmetic).
+
+attention : paper Eq. 3 with the row softmax of Eq. 4 (keys up to the query's own token),
+            evaluated per (row, head) in fp64 by the C routine.
+merge     : the online-softmax combination of two partial results over disjoint key sets
+            (Section 2.2; the colocation example's step 5 in Section 5.2 merges two such
+            partial outputs of one request).
+planner   : integer rules for zigzag sequence partitions, preemptible chunks and causal
+            tile classes.  The paper only says that a long input is cut into segments
+            (Section 2.2) and that a prefill pauses between kernels (Section 5.1); the
+            concrete rule below is this library's convention, written here with Python
+            integers only.
+"""
+import ctypes
+import math
+
+import numpy as np
+
+from . import build as _build
+
+SKIP, PARTIAL, FULL = 0, 1, 2
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(_build.build())
+        lib.pec_oracle_attn_rows.restype = ctypes.c_int
+        lib.pec_oracle_attn_rows.argtypes = [
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+            ctypes.c_int, ctypes.c_int, ctypes.c_int,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+            ctypes.c_int, ctypes.c_double, ctypes.c_void_p, ctypes.c_void_p,
+        ]
+        lib.pec_oracle_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def oracle_threads() -> int:
+    """Host threads the C routine runs on."""
+    return int(_load().pec_oracle_threads())
+
+
+def _as_f32(x):
+    """float32 C-contiguous numpy view/copy of a numpy array or a torch CPU tensor."""
+    if hasattr(x, "detach"):  # torch tensor; bf16 -> fp32 is exact
+        import torch
+        x = x.detach().to("cpu").to(torch.float32).contiguous().numpy()
+    return np.ascontiguousarray(x, dtype=np.float32)
+
+
+# --------------------------------------------------------------------------- planner
+def _ceil_div(a: int, b: int) -> int:
+    return -((-a) // b)
+
+
+def plan_partitions(seq_len, num_parts, chunk_len, align, block_m, block_n, causal, tiles=True):
+    """Zigzag partitions, chunk list, tile classes and visible-pair counts (all Python ints).
+
+    With U = ceil(S/align) alignment units, the sequence is cut into 2P blocks at
+    bounds[k] = min(S, align * floor(k*U / (2P))); partition p owns blocks p and 2P-1-p,
+    which pairs an early (cheap under a causal mask) block with a late (expensive) one.
+    Chunk c covers query rows [c*C, min(S, (c+1)*C)).  A (query tile, key tile) pair is
+    SKIP when every key lies after every query, FULL when no key lies after any query,
+    PARTIAL otherwise; without the causal mask every pair is FULL.  pairs[p] counts the
+    (query, key) pairs partition p's keys contribute when all S rows are queries.
+    """
+    S, P, C = int(seq_len), int(num_parts), int(chunk_len)
+    if S < 0 or P < 1 or align < 1 or block_m < 1 or block_n < 1:
+        raise ValueError("bad planner arguments")
+    if C <= 0:
+        C = max(S, 1)
+    U = _ceil_div(S, align)
+    bounds = [min(S, align * ((k * U) // (2 * P))) for k in range(2 * P + 1)]
+    parts = []
+    pairs = []
+    for p in range(P):
+        ivs = [(bounds[p], bounds[p + 1]), (bounds[2 * P - 1 - p], bounds[2 * P - p])]
+        parts.append(ivs)
+        n = 0
+        for lo, hi in ivs:
+            for j in range(lo, hi):
+                n += (S - j) if causal else S
+        pairs.append(n)
+    n_chunks = _ceil_div(S, C)
+    chunks = [(c * C, min(S, (c + 1) * C) - c * C) for c in range(n_chunks)]
+    nq, nk = _ceil_div(S, block_m), _ceil_div(S, block_n)
+    tile_class = None
+    if tiles:
+        tile_class = np.zeros((nq, nk), dtype=np.uint8)
+        for a in range(nq):
+            q0, q1 = a * block_m, min(S, (a + 1) * block_m)
+            for b in range(nk):
+                k0, k1 = b * block_n, min(S, (b + 1) * block_n)
+                if not causal:
+                    cls = FULL
+                elif k0 > q1 - 1:
+                    cls = SKIP
+                elif k1 - 1 <= q0:
+                    cls = FULL
+                else:
+                    cls = PARTIAL
+                tile_class[a, b] = cls
+    return {
+        "bounds": bounds, "parts": parts, "pairs": pairs, "chunks": chunks,
+        "nq_tiles": nq, "nk_tiles": nk, "tile_class": tile_class,
+    }
+
+
+def partition_intervals(seq_len, num_parts, part_id, align, kv_len=None):
+    """Key intervals of one partition, cut to the available K/V prefix [0, kv_len)."""
+    S, P, p = int(seq_len), int(num_parts), int(part_id)
+    kv_len = S if kv_len is None else int(kv_len)
+    if P == 1:
+        ivs = [(0, S)]
+    else:
+        ivs = plan_partitions(S, P, 0, align, 1, 1, True, tiles=False)["parts"][p]
+    out = []
+    for lo, hi in ivs:
+        hi = min(hi, kv_len)
+        if hi > lo:
+            out.append((lo, hi))
+    return out
+
+
+# --------------------------------------------------------------------------- attention
+def attn_rows(q_rows, q_pos, k, v, intervals, causal, scale=None):
+    """fp64 partial attention of the given query rows over a key set.
+
+    q_rows [n, Hq, D]; q_pos [n] positions of those rows; k, v [n_keys, Hkv, D];
+    intervals: disjoint half-open key ranges.  Returns (O [n,Hq,D] f64, LSE [n,Hq] f64).
+    """
+    q = _as_f32(q_rows)
+    kk = _as_f32(k)
+    vv = _as_f32(v)
+    n, hq, d = q.shape
+    n_keys, hkv, d2 = kk.shape
+    assert d2 == d and vv.shape == kk.shape
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    pos = np.ascontiguousarray(q_pos, dtype=np.int64)
+    assert pos.shape == (n,)
+    lo = np.ascontiguousarray([a for a, _ in intervals], dtype=np.int64)
+    hi = np.ascontiguousarray([b for _, b in intervals], dtype=np.int64)
+    o = np.empty((n, hq, d), dtype=np.float64)
+    lse = np.empty((n, hq), dtype=np.float64)
+    rc = _load().pec_oracle_attn_rows(
+        q.ctypes.data, pos.ctypes.data, n, kk.ctypes.data, vv.ctypes.data, n_keys,
+        hq, hkv, d, lo.ctypes.data, hi.ctypes.data, len(intervals),
+        1 if causal else 0, float(scale), o.ctypes.data, lse.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"pec_oracle_attn_rows failed: {rc}")
+    return o, lse
+
+
+def prefill_attn(q, k, v, *, seq_len, chunk_start=0, chunk_len=None, kv_len=None,
+                 part_id=0, num_parts=1, part_align=128, causal=True, scale=None, rows=None):
+    """What one partial-prefill call must return, for all chunk rows or for sampled ones.
+
+    q holds the whole request's queries [seq_len, Hq, D] (indexed by position);
+    k, v hold at least the first kv_len keys.  rows (optional) lists positions inside
+    the chunk to evaluate; the result rows follow that list's order.
+    """
+    S = int(seq_len)
+    chunk_len = S - chunk_start if chunk_len is None else int(chunk_len)
+    kv_len = S if kv_len is None else int(kv_len)
+    ivs = partition_intervals(S, num_parts, part_id, part_align, kv_len)
+    if rows is None:
+        pos = np.arange(chunk_start, chunk_start + chunk_len, dtype=np.int64)
+    else:
+        pos = np.asarray(rows, dtype=np.int64)
+        assert ((pos >= chunk_start) & (pos < chunk_start + chunk_len)).all()
+    if hasattr(q, "detach"):
+        import torch
+        q_sel = q[torch.as_tensor(pos)]
+    else:
+        q_sel = np.asarray(q)[pos]
+    return attn_rows(q_sel, pos, k[:kv_len], v[:kv_len], ivs, causal, scale)
+
+
+def varlen_attn(q, k, v, cu_seqlens, causal=True, scale=None):
+    """Packed batch: request r owns rows [cu[r], cu[r+1]) and attends only to itself."""
+    cu = [int(x) for x in cu_seqlens]
+    qf = _as_f32(q)
+    total, hq, d = qf.shape
+    o = np.zeros((total, hq, d), dtype=np.float64)
+    lse = np.full((total, hq), -np.inf, dtype=np.float64)
+    for r in range(len(cu) - 1):
+        a, b = cu[r], cu[r + 1]
+        if b == a:
+            continue
+        pos = np.arange(b - a, dtype=np.int64)
+        o[a:b], lse[a:b] = attn_rows(qf[a:b], pos, k[a:b], v[a:b], [(0, b - a)], causal, scale)
+    return o, lse
+
+
+# --------------------------------------------------------------------------- merge
+def merge(o_a, lse_a, o_b, lse_b):
+    """Combine two partial results over disjoint key sets (fp64 numpy).
+
+    LSE = logaddexp(LSE_a, LSE_b); O = e^{LSE_a-LSE} O_a + e^{LSE_b-LSE} O_b.
+    A side with LSE = -inf contributes nothing; both -inf gives (0, -inf).
+    """
+    o_a = np.asarray(o_a, dtype=np.float64)
+    o_b = np.asarray(o_b, dtype=np.float64)
+    la = np.asarray(lse_a, dtype=np.float64)
+    lb = np.asarray(lse_b, dtype=np.float64)
+    m = np.maximum(la, lb)
+    both_empty = np.isneginf(m)
+    m_safe = np.where(both_empty, 0.0, m)
+    wa = np.exp(la - m_safe)
+    wb = np.exp(lb - m_safe)
+    tot = wa + wb
+    lse = np.where(both_empty, -np.inf, m_safe + np.log(np.where(both_empty, 1.0, tot)))
+    ca = np.where(both_empty, 0.0, wa / np.where(both_empty, 1.0, tot))
+    cb = np.where(both_empty, 0.0, wb / np.where(both_empty, 1.0, tot))
+    o = ca[..., None] * o_a + cb[..., None] * o_b
+    return o, lse
