@@ -1,0 +1,174 @@
+/*
+ * pec.h - C ABI of the partial causal prefill attention library (sm_100a).
+ *
+ * The library computes the attention step that PecSched's fast sequence
+ * parallelism and prefill preemption revolve around (arXiv 2409.15104):
+ * causal softmax attention (Eq. 3, with the row softmax of Eq. 4 summing over
+ * the keys up to and including the row's own token) evaluated as a *partial*
+ * result over a subset of the keys, with the per-row log-sum-exp kept so that
+ * partials over disjoint key subsets can be merged exactly (the online-softmax
+ * combination that ring attention relies on, Section 2.2) and so that a
+ * preempted prefill can resume chunk by chunk from its stored K/V prefix
+ * (Section 5.1).
+ *
+ * Conventions for every call:
+ *   - returns PEC_OK (0) or a negative pec_status; never throws, never aborts;
+ *   - never allocates or frees device memory and never synchronises: kernels
+ *     are enqueued on the caller's CUDA stream (`cuda_stream` is a
+ *     cudaStream_t passed as void*, NULL = the legacy default stream);
+ *   - the caller owns every buffer; outputs are undefined after an error;
+ *   - pointers marked "device" must be device-accessible, "host" host memory.
+ */
+#ifndef PEC_H_
+#define PEC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PEC_OK = 0,
+    PEC_ERR_INVALID_ARG = -1, /* NULL pointer, negative size, inconsistent ranges      */
+    PEC_ERR_UNSUPPORTED = -2, /* head_dim != 128, dtype combination not implemented   */
+    PEC_ERR_ALIGNMENT = -3,   /* pointer or stride not aligned as required             */
+    PEC_ERR_WORKSPACE = -4,   /* workspace smaller than pec_workspace_size()           */
+    PEC_ERR_CUDA = -5,        /* a CUDA runtime/driver call or the launch failed       */
+    PEC_ERR_TIMEOUT = -6,     /* value a kernel stores in *status when a bounded wait  */
+                              /* inside it gave up (read it after synchronising)       */
+    PEC_ERR_CAPACITY = -7     /* a caller array of pec_plan is too small               */
+} pec_status;
+
+typedef enum { PEC_BF16 = 1, PEC_F32 = 2 } pec_dtype;
+
+/* Tile classes written by pec_plan_partitions. */
+enum { PEC_TILE_SKIP = 0, PEC_TILE_PARTIAL = 1, PEC_TILE_FULL = 2 };
+
+/*
+ * Arguments of pec_prefill_attn.
+ *
+ * Layout: q is [Tq, Hq, D], k and v are [Tk, Hkv, D] with D contiguous; token
+ * and head strides are given in elements.  Query head h reads KV head
+ * h / (Hq / Hkv) (grouped-query attention, Section 5.3).  D must be 128.
+ *
+ * Single request (cu_seqlens == NULL): row t of q/k/v is the token at position
+ * t of a request of `seq_len` tokens.  The call handles query rows
+ * [chunk_start, chunk_start + chunk_len) and may read keys [0, kv_len) only:
+ * this is one preemptible chunk resumed from the stored K/V prefix
+ * (Section 5.1).  Output row r of o / lse belongs to position chunk_start + r.
+ *
+ * Packed batch (cu_seqlens != NULL): request b owns rows
+ * [cu_seqlens[b], cu_seqlens[b+1]) of q, k, v, o and lse and attends only to
+ * itself, each request starting at position 0 (short-request batches,
+ * Section 5.2).  seq_len is the total number of packed rows (cu_seqlens[B]),
+ * chunk_start must be 0, chunk_len and kv_len must equal seq_len, num_parts
+ * must be 1.
+ *
+ * Key subset: with num_parts == 1 all keys of [0, kv_len); otherwise zigzag
+ * partition part_id of num_parts as defined by pec_plan_partitions(seq_len,
+ * num_parts, ..., part_align, ...), intersected with [0, kv_len).  With
+ * `causal`, key j is visible to the query at position i iff j <= i.
+ *
+ * Results: o[r, h, :] = sum_j p_j v_j over the visible keys of the subset with
+ * p the softmax of softmax_scale * q.k restricted to that subset, and
+ * lse[r, h] = ln sum_j exp(softmax_scale * q.k_j) (natural log, fp32).  A row
+ * with no visible key gets o = 0 and lse = -inf, the identity of
+ * pec_attn_merge.  o_dtype PEC_F32 gives a partial fit for merging;
+ * PEC_BF16 rounds to nearest-even (allowed with in_dtype PEC_BF16 only).
+ *
+ * in_dtype PEC_BF16 runs the tcgen05 tensor-core kernel (bf16 products, fp32
+ * accumulation); PEC_F32 runs an fp32 FMA kernel (accuracy path).
+ */
+typedef struct {
+    const void *q, *k, *v;      /* device; 16-byte aligned                              */
+    int64_t q_stride_t, q_stride_h;
+    int64_t k_stride_t, k_stride_h;
+    int64_t v_stride_t, v_stride_h;   /* elements; bf16: multiples of 8               */
+    int32_t in_dtype;           /* pec_dtype of q, k, v                                  */
+    void *o;                    /* device; [rows, Hq, D] contiguous, 16-byte aligned     */
+    int32_t o_dtype;            /* pec_dtype of o                                        */
+    float *lse;                 /* device; [rows, Hq] contiguous                         */
+    int32_t Hq, Hkv, D;
+    const int32_t *cu_seqlens;  /* device; [B+1] non-decreasing, or NULL                 */
+    int32_t B;                  /* number of packed requests (ignored when NULL above)   */
+    int64_t seq_len;
+    int64_t chunk_start, chunk_len;
+    int64_t kv_len;             /* causal calls need kv_len >= chunk_start + chunk_len   */
+    int32_t part_id, num_parts;
+    int32_t part_align;         /* partition alignment in tokens (>= 1)                  */
+    int32_t causal;             /* 0 or 1                                                */
+    float softmax_scale;        /* 0 selects 1/sqrt(D)                                   */
+    void *workspace;            /* device scratch of pec_workspace_size() bytes or NULL  */
+    size_t workspace_bytes;
+    int32_t *status;            /* device word, may be NULL; the caller zeroes it; a     */
+                                /* kernel stores PEC_ERR_TIMEOUT there if a wait expired */
+} pec_attn_args;
+
+/*
+ * Partial attention of one chunk / partition / packed batch (Eq. 3-4; see the
+ * struct above).  Validates the arguments on the host, then enqueues one kernel.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.
+ */
+int pec_prefill_attn(const pec_attn_args *args, void *cuda_stream);
+
+/* Bytes of device scratch pec_prefill_attn needs for these arguments (may be 0). */
+size_t pec_workspace_size(const pec_attn_args *args);
+
+/*
+ * Merge two partial results of the same rows over disjoint key subsets
+ * (online-softmax combination, Section 2.2; the two-GPU outputs O_1, O_2 of one
+ * request in Section 5.2's colocation example are combined this way):
+ *     lse = ln(exp(lse_a) + exp(lse_b))
+ *     o   = exp(lse_a - lse) * o_a + exp(lse_b - lse) * o_b
+ * per (row, head); a side with lse = -inf contributes nothing, both -inf give
+ * o = 0, lse = -inf.  o_a, o_b: device [rows, Hq, D] fp32 (part_dtype must be
+ * PEC_F32); lse_*: device [rows, Hq] fp32; o_out: device [rows, Hq, D] of
+ * out_dtype (PEC_F32 or PEC_BF16); all contiguous and 16-byte aligned.  o_out /
+ * lse_out may alias o_a / lse_a (running merge) when out_dtype == PEC_F32.
+ * D must be 128.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.
+ */
+int pec_attn_merge(const void *o_a, const float *lse_a, const void *o_b, const float *lse_b,
+                   void *o_out, float *lse_out, int64_t rows, int32_t Hq, int32_t D,
+                   int32_t part_dtype, int32_t out_dtype, void *cuda_stream);
+
+/*
+ * Host-side plan of how a request of seq_len tokens is split.  All arrays are
+ * host memory owned by the caller; an array pointer may be NULL to skip that
+ * output.  Capacities are element counts; the needed counts are always written
+ * to the n_* fields, so a first call with NULL arrays is a size query.
+ *
+ * The paper cuts a long input into segments handled by different replicas
+ * (Section 2.2) and pauses a prefill between kernels (Section 5.1) without
+ * fixing either rule; this library's integer rule is:
+ *   U = ceil(seq_len / align);  bounds[k] = min(seq_len, align * floor(k*U / (2P))), k = 0..2P
+ *   block k = [bounds[k], bounds[k+1]);  partition p owns blocks p and 2P-1-p (zigzag)
+ *   part_lo/part_hi[2p], [2p+1] = those two intervals (an interval may be empty)
+ *   pairs[p] = number of (query, key) pairs with the key in partition p, over all
+ *              seq_len query rows: sum (seq_len - j) if causal, else seq_len per key
+ *   chunk c = [c*chunk_len, min(seq_len, (c+1)*chunk_len));  chunk_len <= 0: one chunk
+ *   tile_class[a*nk_tiles + b] for query tile a (block_m rows) and key tile b
+ *   (block_n keys): causal: SKIP if the tile's first key is after its last query,
+ *   FULL if its last key is not after its first query, else PARTIAL; non-causal: FULL.
+ */
+typedef struct {
+    int64_t *bounds;      int64_t bounds_cap;  /* 2P+1                      */
+    int64_t *part_lo;     int64_t *part_hi;    int64_t part_cap;   /* 2P    */
+    int64_t *pairs;       int64_t pairs_cap;   /* P                         */
+    int64_t *chunk_start; int64_t *chunk_len;  int64_t chunk_cap;  /* n_chunks */
+    uint8_t *tile_class;  int64_t tile_cap;    /* nq_tiles * nk_tiles       */
+    int64_t n_bounds, n_parts, n_chunks, nq_tiles, nk_tiles;       /* outputs */
+} pec_plan;
+
+/* Errors: INVALID_ARG (seq_len < 0, num_parts < 1, align/block < 1, NULL plan), CAPACITY. */
+int pec_plan_partitions(int64_t seq_len, int32_t num_parts, int64_t chunk_len, int32_t align,
+                        int32_t block_m, int32_t block_n, int32_t causal, pec_plan *plan);
+
+/* Text describing the last non-zero return on this thread (never NULL). */
+const char *pec_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PEC_H_ */

@@ -1,0 +1,243 @@
+"""ctypes binding of libpec.so.  Argument marshalling only: every step runs in the library.
+
+Function names mirror the C ABI (include/pec.h).  torch provides device memory and streams.
+The library is loaded on first use; a missing or unloadable library raises - there is no
+fallback implementation.
+"""
+import ctypes
+import os
+
+import torch
+
+PEC_OK = 0
+PEC_ERR_TIMEOUT = -6
+PEC_BF16, PEC_F32 = 1, 2
+PEC_TILE_SKIP, PEC_TILE_PARTIAL, PEC_TILE_FULL = 0, 1, 2
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpec.so")
+_lib = None
+_status_words = {}
+
+
+class PecError(RuntimeError):
+    def __init__(self, code, text):
+        super().__init__(f"pec error {code}: {text}")
+        self.code = code
+
+
+class pec_attn_args(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
+        ("q_stride_t", ctypes.c_int64), ("q_stride_h", ctypes.c_int64),
+        ("k_stride_t", ctypes.c_int64), ("k_stride_h", ctypes.c_int64),
+        ("v_stride_t", ctypes.c_int64), ("v_stride_h", ctypes.c_int64),
+        ("in_dtype", ctypes.c_int32),
+        ("o", ctypes.c_void_p), ("o_dtype", ctypes.c_int32),
+        ("lse", ctypes.c_void_p),
+        ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32),
+        ("cu_seqlens", ctypes.c_void_p), ("B", ctypes.c_int32),
+        ("seq_len", ctypes.c_int64),
+        ("chunk_start", ctypes.c_int64), ("chunk_len", ctypes.c_int64),
+        ("kv_len", ctypes.c_int64),
+        ("part_id", ctypes.c_int32), ("num_parts", ctypes.c_int32),
+        ("part_align", ctypes.c_int32), ("causal", ctypes.c_int32),
+        ("softmax_scale", ctypes.c_float),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+        ("status", ctypes.c_void_p),
+    ]
+
+
+class pec_plan(ctypes.Structure):
+    _fields_ = [
+        ("bounds", ctypes.POINTER(ctypes.c_int64)), ("bounds_cap", ctypes.c_int64),
+        ("part_lo", ctypes.POINTER(ctypes.c_int64)), ("part_hi", ctypes.POINTER(ctypes.c_int64)),
+        ("part_cap", ctypes.c_int64),
+        ("pairs", ctypes.POINTER(ctypes.c_int64)), ("pairs_cap", ctypes.c_int64),
+        ("chunk_start", ctypes.POINTER(ctypes.c_int64)), ("chunk_len", ctypes.POINTER(ctypes.c_int64)),
+        ("chunk_cap", ctypes.c_int64),
+        ("tile_class", ctypes.POINTER(ctypes.c_uint8)), ("tile_cap", ctypes.c_int64),
+        ("n_bounds", ctypes.c_int64), ("n_parts", ctypes.c_int64), ("n_chunks", ctypes.c_int64),
+        ("nq_tiles", ctypes.c_int64), ("nk_tiles", ctypes.c_int64),
+    ]
+
+
+EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_plan_partitions", "pec_last_error")
+
+
+def load():
+    """Load libpec.so (building is a separate step: python -m paper_2409_15104_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2409_15104_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    lib.pec_prefill_attn.restype = ctypes.c_int
+    lib.pec_prefill_attn.argtypes = [ctypes.POINTER(pec_attn_args), ctypes.c_void_p]
+    lib.pec_workspace_size.restype = ctypes.c_size_t
+    lib.pec_workspace_size.argtypes = [ctypes.POINTER(pec_attn_args)]
+    lib.pec_attn_merge.restype = ctypes.c_int
+    lib.pec_attn_merge.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32,
+                                   ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
+    lib.pec_plan_partitions.restype = ctypes.c_int
+    lib.pec_plan_partitions.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, ctypes.c_int32,
+                                        ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(pec_plan)]
+    lib.pec_last_error.restype = ctypes.c_char_p
+    lib.pec_last_error.argtypes = []
+    _lib = lib
+    return lib
+
+
+def pec_last_error() -> str:
+    return load().pec_last_error().decode()
+
+
+def _check(rc):
+    if rc != PEC_OK:
+        raise PecError(rc, pec_last_error())
+
+
+def _dtype_code(dt):
+    if dt == torch.bfloat16:
+        return PEC_BF16
+    if dt == torch.float32:
+        return PEC_F32
+    raise TypeError(f"unsupported dtype {dt}")
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def status_word(device=None) -> torch.Tensor:
+    """The per-device int32 word kernels flag expired waits in (zero = fine)."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+    key = dev.index if dev.index is not None else torch.cuda.current_device()
+    if key not in _status_words:
+        _status_words[key] = torch.zeros(1, dtype=torch.int32, device=dev)
+    return _status_words[key]
+
+
+def check_status(device=None):
+    """Synchronise and raise if a kernel recorded an expired wait; clears the word."""
+    w = status_word(device)
+    code = int(w.item())
+    if code != 0:
+        w.zero_()
+        raise PecError(code, "a kernel's bounded wait expired" if code == PEC_ERR_TIMEOUT else "kernel status")
+
+
+def pec_prefill_attn(q, k, v, *, seq_len=None, chunk_start=0, chunk_len=None, kv_len=None,
+                     part_id=0, num_parts=1, part_align=128, causal=True, softmax_scale=0.0,
+                     cu_seqlens=None, out_dtype=None, o=None, lse=None, stream=None):
+    """Partial attention of one chunk / partition / packed batch; returns (o, lse).
+
+    q [T, Hq, 128], k / v [Tk, Hkv, 128] CUDA tensors (last dim contiguous).  Single request:
+    rows are positions, the call covers query rows [chunk_start, chunk_start+chunk_len) against
+    keys [0, kv_len).  Packed batch: pass cu_seqlens (int32 CUDA tensor [B+1]).
+    o / lse may be passed in (views are fine as long as they are contiguous).
+    """
+    lib = load()
+    assert q.is_cuda and k.is_cuda and v.is_cuda
+    assert q.stride(2) == 1 and k.stride(2) == 1 and v.stride(2) == 1
+    T, Hq, D = q.shape
+    Hkv = k.shape[1]
+    if cu_seqlens is not None:
+        B = cu_seqlens.numel() - 1
+        seq_len = T if seq_len is None else seq_len
+        chunk_len = seq_len
+        kv_len = seq_len
+    else:
+        B = 1
+        seq_len = T if seq_len is None else seq_len
+        chunk_len = seq_len - chunk_start if chunk_len is None else chunk_len
+        kv_len = (chunk_start + chunk_len if causal else seq_len) if kv_len is None else kv_len
+    out_dtype = (torch.float32 if num_parts > 1 else q.dtype) if out_dtype is None else out_dtype
+    if o is None:
+        o = torch.empty((chunk_len, Hq, D), dtype=out_dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((chunk_len, Hq), dtype=torch.float32, device=q.device)
+    assert o.is_contiguous() and lse.is_contiguous() and lse.dtype == torch.float32
+    a = pec_attn_args()
+    a.q, a.k, a.v = q.data_ptr(), k.data_ptr(), v.data_ptr()
+    a.q_stride_t, a.q_stride_h = q.stride(0), q.stride(1)
+    a.k_stride_t, a.k_stride_h = k.stride(0), k.stride(1)
+    a.v_stride_t, a.v_stride_h = v.stride(0), v.stride(1)
+    a.in_dtype = _dtype_code(q.dtype)
+    a.o, a.o_dtype, a.lse = o.data_ptr(), _dtype_code(o.dtype), lse.data_ptr()
+    a.Hq, a.Hkv, a.D = Hq, Hkv, D
+    a.cu_seqlens = cu_seqlens.data_ptr() if cu_seqlens is not None else None
+    a.B = B
+    a.seq_len, a.chunk_start, a.chunk_len, a.kv_len = seq_len, chunk_start, chunk_len, kv_len
+    a.part_id, a.num_parts, a.part_align = part_id, num_parts, part_align
+    a.causal = 1 if causal else 0
+    a.softmax_scale = float(softmax_scale)
+    a.workspace, a.workspace_bytes = None, 0
+    a.status = status_word(q.device).data_ptr()
+    _check(lib.pec_prefill_attn(ctypes.byref(a), _stream_ptr(stream)))
+    return o, lse
+
+
+def pec_workspace_size(**kw) -> int:
+    a = pec_attn_args()
+    for key, val in kw.items():
+        setattr(a, key, val)
+    return int(load().pec_workspace_size(ctypes.byref(a)))
+
+
+def pec_attn_merge(o_a, lse_a, o_b, lse_b, *, out_dtype=torch.float32, o_out=None, lse_out=None,
+                   inplace=False, stream=None):
+    """Merge two fp32 partials of the same rows; returns (o, lse).  inplace=True writes into side a."""
+    lib = load()
+    rows, Hq, D = o_a.shape
+    for t in (o_a, lse_a, o_b, lse_b):
+        assert t.is_cuda and t.is_contiguous()
+    if inplace:
+        o_out, lse_out = o_a, lse_a
+    if o_out is None:
+        o_out = torch.empty((rows, Hq, D), dtype=out_dtype, device=o_a.device)
+    if lse_out is None:
+        lse_out = torch.empty((rows, Hq), dtype=torch.float32, device=o_a.device)
+    _check(lib.pec_attn_merge(o_a.data_ptr(), lse_a.data_ptr(), o_b.data_ptr(), lse_b.data_ptr(),
+                              o_out.data_ptr(), lse_out.data_ptr(), rows, Hq, D,
+                              _dtype_code(o_a.dtype), _dtype_code(o_out.dtype), _stream_ptr(stream)))
+    return o_out, lse_out
+
+
+def pec_plan_partitions(seq_len, num_parts, chunk_len=0, align=128, block_m=128, block_n=128,
+                        causal=True, tiles=True):
+    """Host plan (see include/pec.h) as a dict of Python ints / a numpy uint8 tile-class array."""
+    import numpy as np
+    lib = load()
+    plan = pec_plan()
+    _check(lib.pec_plan_partitions(seq_len, num_parts, chunk_len, align, block_m, block_n, 1 if causal else 0,
+                                   ctypes.byref(plan)))
+    P, nch = plan.n_parts, plan.n_chunks
+    bounds = (ctypes.c_int64 * plan.n_bounds)()
+    lo = (ctypes.c_int64 * (2 * P))()
+    hi = (ctypes.c_int64 * (2 * P))()
+    pairs = (ctypes.c_int64 * P)()
+    cs = (ctypes.c_int64 * max(nch, 1))()
+    cl = (ctypes.c_int64 * max(nch, 1))()
+    plan.bounds, plan.bounds_cap = bounds, plan.n_bounds
+    plan.part_lo, plan.part_hi, plan.part_cap = lo, hi, 2 * P
+    plan.pairs, plan.pairs_cap = pairs, P
+    plan.chunk_start, plan.chunk_len, plan.chunk_cap = cs, cl, max(nch, 1)
+    tc = None
+    if tiles:
+        tc = np.zeros((plan.nq_tiles, plan.nk_tiles), dtype=np.uint8)
+        plan.tile_class = tc.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8))
+        plan.tile_cap = tc.size
+    _check(lib.pec_plan_partitions(seq_len, num_parts, chunk_len, align, block_m, block_n, 1 if causal else 0,
+                                   ctypes.byref(plan)))
+    return {
+        "bounds": [int(x) for x in bounds],
+        "parts": [[(int(lo[2 * p]), int(hi[2 * p])), (int(lo[2 * p + 1]), int(hi[2 * p + 1]))] for p in range(P)],
+        "pairs": [int(x) for x in pairs],
+        "chunks": [(int(cs[c]), int(cl[c])) for c in range(nch)],
+        "nq_tiles": int(plan.nq_tiles), "nk_tiles": int(plan.nk_tiles), "tile_class": tc,
+    }

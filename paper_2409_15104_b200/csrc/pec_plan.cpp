@@ -1,0 +1,107 @@
+// Host planner: zigzag sequence partitions, preemptible chunks, causal tile classes.
+// Integer arithmetic only; the rule is stated in pec.h.  The paper asks for segments handled
+// by different replicas (Section 2.2) and for prefills that pause between kernels
+// (Section 5.1); pairing block p with block 2P-1-p equalises the causal work per partition.
+#include "pec_internal.h"
+
+namespace pec {
+
+static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+static inline int64_t bound_at(int64_t k, int64_t units, int64_t two_p, int64_t align, int64_t seq_len)
+{
+    // k <= 2P and units <= 2^63 / (2P) for any realistic length: the product fits in int64.
+    const int64_t b = align * ((k * units) / two_p);
+    return b < seq_len ? b : seq_len;
+}
+
+void zigzag_intervals(int64_t seq_len, int32_t num_parts, int32_t part_id, int32_t align,
+                      int64_t lo[2], int64_t hi[2])
+{
+    const int64_t two_p = 2 * (int64_t)num_parts;
+    const int64_t units = ceil_div(seq_len, align);
+    const int64_t a = part_id, b = two_p - 1 - part_id;
+    lo[0] = bound_at(a, units, two_p, align, seq_len);
+    hi[0] = bound_at(a + 1, units, two_p, align, seq_len);
+    lo[1] = bound_at(b, units, two_p, align, seq_len);
+    hi[1] = bound_at(b + 1, units, two_p, align, seq_len);
+}
+
+}  // namespace pec
+
+using namespace pec;
+
+extern "C" int pec_plan_partitions(int64_t seq_len, int32_t num_parts, int64_t chunk_len, int32_t align,
+                                   int32_t block_m, int32_t block_n, int32_t causal, pec_plan *plan)
+{
+    if (!plan) { set_error("pec_plan_partitions: plan is NULL"); return PEC_ERR_INVALID_ARG; }
+    if (seq_len < 0 || num_parts < 1 || align < 1 || block_m < 1 || block_n < 1) {
+        set_error("pec_plan_partitions: need seq_len >= 0, num_parts >= 1, align >= 1, block_m/n >= 1");
+        return PEC_ERR_INVALID_ARG;
+    }
+    const int64_t P = num_parts, two_p = 2 * P;
+    const int64_t units = ceil_div(seq_len, align);
+    const int64_t C = chunk_len > 0 ? chunk_len : (seq_len > 0 ? seq_len : 1);
+    plan->n_bounds = two_p + 1;
+    plan->n_parts = P;
+    plan->n_chunks = ceil_div(seq_len, C);
+    plan->nq_tiles = ceil_div(seq_len, block_m);
+    plan->nk_tiles = ceil_div(seq_len, block_n);
+
+    if ((plan->bounds && plan->bounds_cap < plan->n_bounds) ||
+        ((plan->part_lo || plan->part_hi) && plan->part_cap < two_p) ||
+        (plan->pairs && plan->pairs_cap < P) ||
+        ((plan->chunk_start || plan->chunk_len) && plan->chunk_cap < plan->n_chunks) ||
+        (plan->tile_class && plan->tile_cap < plan->nq_tiles * plan->nk_tiles)) {
+        set_error("pec_plan_partitions: a caller array is smaller than the count it must hold");
+        return PEC_ERR_CAPACITY;
+    }
+
+    if (plan->bounds)
+        for (int64_t k = 0; k <= two_p; ++k) plan->bounds[k] = bound_at(k, units, two_p, align, seq_len);
+
+    for (int64_t p = 0; p < P; ++p) {
+        int64_t lo[2], hi[2];
+        zigzag_intervals(seq_len, num_parts, (int32_t)p, align, lo, hi);
+        if (plan->part_lo) { plan->part_lo[2 * p] = lo[0]; plan->part_lo[2 * p + 1] = lo[1]; }
+        if (plan->part_hi) { plan->part_hi[2 * p] = hi[0]; plan->part_hi[2 * p + 1] = hi[1]; }
+        if (plan->pairs) {
+            // sum_{j=lo}^{hi-1} (S - j) = n*S - (lo + hi - 1)*n/2, kept exact in 128-bit.
+            __int128 total = 0;
+            for (int t = 0; t < 2; ++t) {
+                const __int128 n = hi[t] - lo[t];
+                if (n <= 0) continue;
+                if (causal) total += n * seq_len - ((__int128)(lo[t] + hi[t] - 1) * n) / 2;
+                else        total += n * seq_len;
+            }
+            plan->pairs[p] = (int64_t)total;
+        }
+    }
+
+    for (int64_t c = 0; c < plan->n_chunks; ++c) {
+        const int64_t s = c * C;
+        const int64_t e = (s + C < seq_len) ? s + C : seq_len;
+        if (plan->chunk_start) plan->chunk_start[c] = s;
+        if (plan->chunk_len) plan->chunk_len[c] = e - s;
+    }
+
+    if (plan->tile_class) {
+        for (int64_t a = 0; a < plan->nq_tiles; ++a) {
+            const int64_t q0 = a * block_m;
+            const int64_t q1 = (q0 + block_m < seq_len) ? q0 + block_m : seq_len;   // exclusive
+            uint8_t *row = plan->tile_class + a * plan->nk_tiles;
+            for (int64_t b = 0; b < plan->nk_tiles; ++b) {
+                const int64_t k0 = b * block_n;
+                const int64_t k1 = (k0 + block_n < seq_len) ? k0 + block_n : seq_len;
+                uint8_t cls = PEC_TILE_FULL;
+                if (causal) {
+                    if (k0 > q1 - 1) cls = PEC_TILE_SKIP;
+                    else if (k1 - 1 <= q0) cls = PEC_TILE_FULL;
+                    else cls = PEC_TILE_PARTIAL;
+                }
+                row[b] = cls;
+            }
+        }
+    }
+    return PEC_OK;
+}

@@ -1,0 +1,54 @@
+// Device-side mapping from a linear tile index to the rows and key intervals it covers.
+#pragma once
+#include "pec_internal.h"
+
+namespace pec {
+
+struct TileJob {
+    int64_t q_row0;      // first row of the tile in q
+    int64_t out_row0;    // first row of the tile in o / lse
+    int64_t q_pos0;      // position of that row in its request
+    int32_t n_rows;      // valid rows in the tile
+    int64_t kv_row0;     // row of key position 0 in k / v
+    int64_t iv_lo[2], iv_hi[2];   // visible-key intervals (positions), before the causal cut
+    int32_t n_iv;
+};
+
+// Returns false when `tile` is past the last tile.  Packed batches walk cu_seqlens: request b
+// contributes ceil(len_b / block_m) tiles, each request starting a fresh tile.
+__device__ __forceinline__ bool locate_tile(const AttnParams &p, int64_t tile, int block_m, TileJob &job)
+{
+    if (p.cu_seqlens == nullptr) {
+        const int64_t r0 = tile * block_m;
+        if (r0 >= p.chunk_len) return false;
+        job.q_row0 = p.chunk_start + r0;
+        job.out_row0 = r0;
+        job.q_pos0 = p.chunk_start + r0;
+        job.n_rows = (int32_t)((p.chunk_len - r0) < block_m ? (p.chunk_len - r0) : block_m);
+        job.kv_row0 = 0;
+        job.n_iv = p.n_iv;
+        for (int t = 0; t < 2; ++t) { job.iv_lo[t] = p.iv_lo[t]; job.iv_hi[t] = p.iv_hi[t]; }
+        return true;
+    }
+    int64_t t = tile;
+    for (int b = 0; b < p.B; ++b) {
+        const int64_t s = p.cu_seqlens[b], e = p.cu_seqlens[b + 1];
+        const int64_t nt = (e - s + block_m - 1) / block_m;
+        if (t < nt) {
+            const int64_t r0 = t * block_m;
+            job.q_row0 = s + r0;
+            job.out_row0 = s + r0;
+            job.q_pos0 = r0;
+            job.n_rows = (int32_t)((e - s - r0) < block_m ? (e - s - r0) : block_m);
+            job.kv_row0 = s;
+            job.n_iv = 1;
+            job.iv_lo[0] = 0; job.iv_hi[0] = e - s;
+            job.iv_lo[1] = 0; job.iv_hi[1] = 0;
+            return true;
+        }
+        t -= nt;
+    }
+    return false;
+}
+
+}  // namespace pec

@@ -1,0 +1,189 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle, element by element,
+at sizes that span several tiles and ragged tails, plus the degenerate cases."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import TOL, compare
+from paper_2409_15104_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _qkv(seed, T, hq, hkv, dtype):
+    q, k, v = workloads.qkv(seed, T, hq, hkv, 128, dtype)
+    return q, k, v
+
+
+def _gpu(*ts):
+    return [t.to(DEV) for t in ts]
+
+
+# ------------------------------------------------------------------ merge kernel
+@pytest.mark.parametrize("rows,hq", [(1, 1), (33, 3), (1000, 8), (4096, 32), (77, 5)])
+@pytest.mark.parametrize("mode", ["f32", "bf16", "inplace"])
+def test_merge_matches_oracle(pec, rows, hq, mode):
+    g = torch.Generator().manual_seed(rows * 131 + hq)
+    oa, ob = torch.randn(rows, hq, 128, generator=g), torch.randn(rows, hq, 128, generator=g)
+    la, lb = torch.randn(rows, hq, generator=g) * 4, torch.randn(rows, hq, generator=g) * 4
+    # empty sides: a only, b only, both
+    la[0::7] = float("-inf"); oa[0::7] = 0
+    lb[3::5] = float("-inf"); ob[3::5] = 0
+    want_o, want_l = oracle.merge(oa.numpy(), la.numpy(), ob.numpy(), lb.numpy())
+    doa, dla, dob, dlb = _gpu(oa, la, ob, lb)
+    if mode == "inplace":
+        o, l = pec.pec_attn_merge(doa, dla, dob, dlb, inplace=True)
+        assert o.data_ptr() == doa.data_ptr()
+    else:
+        o, l = pec.pec_attn_merge(doa, dla, dob, dlb, out_dtype=torch.float32 if mode == "f32" else torch.bfloat16)
+    tol_o = 2e-2 if mode == "bf16" else 1e-5
+    compare(o, l, want_o, want_l, tol_o, 1e-5, f"merge {mode}")
+
+
+def test_merge_ignores_garbage_behind_an_empty_side(pec):
+    rows, hq = 64, 4
+    oa = torch.randn(rows, hq, 128); la = torch.randn(rows, hq)
+    ob = torch.full((rows, hq, 128), float("nan")); lb = torch.full((rows, hq), float("-inf"))
+    o, l = pec.pec_attn_merge(*_gpu(oa, la, ob, lb))
+    assert torch.equal(o.cpu(), oa) and torch.equal(l.cpu(), la)
+
+
+# ------------------------------------------------------------------ attention, single request
+SHAPES = [  # (S, Hq, Hkv)
+    (1, 1, 1), (2, 2, 1), (63, 2, 2), (64, 4, 2), (65, 2, 1), (127, 4, 4), (128, 8, 2), (129, 2, 2),
+    (255, 4, 1), (257, 2, 2), (384, 8, 8), (1000, 4, 2),
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("S,hq,hkv", SHAPES)
+def test_full_causal_prefill(pec, dtype, S, hq, hkv):
+    q, k, v = _qkv(1000 + S, S, hq, hkv, dtype)
+    want = oracle.prefill_attn(q, k, v, seq_len=S)
+    o, lse = pec.pec_prefill_attn(*_gpu(q, k, v))
+    pec.check_status()
+    assert o.dtype == dtype
+    compare(o, lse, *want, *TOL[dtype], f"causal S={S} {dtype}")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_non_causal(pec, dtype):
+    S = 300
+    q, k, v = _qkv(2000, S, 4, 2, dtype)
+    want = oracle.prefill_attn(q, k, v, seq_len=S, causal=False)
+    o, lse = pec.pec_prefill_attn(*_gpu(q, k, v), causal=False)
+    pec.check_status()
+    compare(o, lse, *want, *TOL[dtype], "non-causal")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("S,P,align", [(1024, 4, 128), (700, 3, 64), (515, 2, 1), (130, 4, 128), (2048, 8, 128)])
+def test_partition_partials_and_their_merge(pec, dtype, S, P, align):
+    q, k, v = _qkv(3000 + S, S, 4, 2, dtype)
+    dq, dk, dv = _gpu(q, k, v)
+    acc = None
+    for p in range(P):
+        want = oracle.prefill_attn(q, k, v, seq_len=S, part_id=p, num_parts=P, part_align=align)
+        o, lse = pec.pec_prefill_attn(dq, dk, dv, part_id=p, num_parts=P, part_align=align)
+        pec.check_status()
+        assert o.dtype == torch.float32
+        compare(o, lse, *want, *TOL[dtype], f"partition {p}/{P} S={S}")
+        acc = (o, lse) if acc is None else pec.pec_attn_merge(*acc, o, lse, inplace=True)
+    full = oracle.prefill_attn(q, k, v, seq_len=S)
+    compare(acc[0], acc[1], *full, *TOL[dtype], f"merged {P} partitions S={S}")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("S,C", [(1000, 256), (777, 100), (512, 128)])
+def test_chunked_prefill_resumes_from_the_kv_prefix(pec, dtype, S, C):
+    q, k, v = _qkv(4000 + S, S, 4, 1, dtype)
+    dq, dk, dv = _gpu(q, k, v)
+    want = oracle.prefill_attn(q, k, v, seq_len=S)
+    o = torch.full((S, 4, 128), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((S, 4), float("nan"), dtype=torch.float32, device=DEV)
+    for c0 in range(0, S, C):
+        n = min(C, S - c0)
+        # K/V beyond the prefix are poisoned: a resumed chunk must not read them
+        kk, vv = dk.clone(), dv.clone()
+        kk[c0 + n:] = float("nan"); vv[c0 + n:] = float("nan")
+        pec.pec_prefill_attn(dq, kk, vv, seq_len=S, chunk_start=c0, chunk_len=n, kv_len=c0 + n,
+                             o=o[c0:c0 + n], lse=lse[c0:c0 + n])
+    pec.check_status()
+    compare(o, lse, *want, *TOL[dtype], f"chunked S={S} C={C}")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_chunk_of_one_partition(pec, dtype):
+    """A middle chunk against one zigzag partition cut by the K/V prefix."""
+    S, P, c0, n = 1024, 4, 384, 200
+    q, k, v = _qkv(5000, S, 2, 2, dtype)
+    for p in range(P):
+        want = oracle.prefill_attn(q, k, v, seq_len=S, chunk_start=c0, chunk_len=n, kv_len=c0 + n,
+                                   part_id=p, num_parts=P)
+        o, lse = pec.pec_prefill_attn(*_gpu(q, k, v), seq_len=S, chunk_start=c0, chunk_len=n, kv_len=c0 + n,
+                                      part_id=p, num_parts=P)
+        pec.check_status()
+        compare(o, lse, *want, *TOL[dtype], f"chunk x partition {p}")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_strided_inputs_and_custom_scale(pec, dtype):
+    """Q/K/V as slices of one fused [T, Hq+2Hkv, 128] projection output."""
+    S, hq, hkv = 200, 4, 2
+    fused = workloads.normal_tensor(6000, 1, (S, hq + 2 * hkv, 128), dtype)
+    q, k, v = fused[:, :hq], fused[:, hq:hq + hkv], fused[:, hq + hkv:]
+    want = oracle.prefill_attn(q, k, v, seq_len=S, scale=0.05)
+    d = fused.to(DEV)
+    o, lse = pec.pec_prefill_attn(d[:, :hq], d[:, hq:hq + hkv], d[:, hq + hkv:], softmax_scale=0.05)
+    pec.check_status()
+    compare(o, lse, *want, *TOL[dtype], "strided")
+
+
+# ------------------------------------------------------------------ packed batches
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("lens", [[5], [128, 128], [1, 300, 0, 77, 129, 64], [200, 1, 1, 511]])
+def test_varlen_batch(pec, dtype, lens):
+    cu = workloads.cu_seqlens(lens)
+    T = cu[-1]
+    q, k, v = _qkv(7000 + T, T, 4, 2, dtype)
+    want = oracle.varlen_attn(q, k, v, cu)
+    dcu = torch.tensor(cu, dtype=torch.int32, device=DEV)
+    o, lse = pec.pec_prefill_attn(*_gpu(q, k, v), cu_seqlens=dcu)
+    pec.check_status()
+    compare(o, lse, *want, *TOL[dtype], f"varlen {lens}")
+
+
+def test_bf16_partial_output_can_stay_fp32_or_round_to_bf16(pec):
+    S = 256
+    q, k, v = _qkv(8000, S, 2, 2, torch.bfloat16)
+    want = oracle.prefill_attn(q, k, v, seq_len=S)
+    o32, l32 = pec.pec_prefill_attn(*_gpu(q, k, v), out_dtype=torch.float32)
+    o16, l16 = pec.pec_prefill_attn(*_gpu(q, k, v), out_dtype=torch.bfloat16)
+    pec.check_status()
+    compare(o32, l32, *want, 2e-2, 1e-3, "fp32 out")
+    compare(o16, l16, *want, 2e-2, 1e-3, "bf16 out")
+    assert torch.equal(l32, l16)
+    assert torch.equal(o32.to(torch.bfloat16), o16)     # same accumulator, rounded once
+
+
+def test_runs_are_bitwise_repeatable(pec):
+    S = 640
+    q, k, v = _gpu(*_qkv(9000, S, 4, 2, torch.bfloat16))
+    a = pec.pec_prefill_attn(q, k, v)
+    b = pec.pec_prefill_attn(q, k, v)
+    pec.check_status()
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+def test_canaries_around_outputs_stay_untouched(pec):
+    S, hq = 333, 2
+    q, k, v = _gpu(*_qkv(9100, S, hq, 1, torch.bfloat16))
+    pad = 64
+    obuf = torch.full(((S + 2 * pad), hq, 128), 7.0, dtype=torch.bfloat16, device=DEV)
+    lbuf = torch.full(((S + 2 * pad), hq), 7.0, dtype=torch.float32, device=DEV)
+    pec.pec_prefill_attn(q, k, v, o=obuf[pad:pad + S], lse=lbuf[pad:pad + S])
+    pec.check_status()
+    assert (obuf[:pad] == 7).all() and (obuf[pad + S:] == 7).all()
+    assert (lbuf[:pad] == 7).all() and (lbuf[pad + S:] == 7).all()

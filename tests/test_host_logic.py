@@ -1,0 +1,111 @@
+"""CPU-only checks of the library's host side: exported symbols, planner parity with the
+oracle (bit-exact), and argument validation (no kernel is launched by these calls)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2409_15104_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = binding.load()
+    header = open(os.path.join(ROOT, "include", "pec.h")).read()
+    declared = set(re.findall(r"\b(pec_[a-z_]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+PLAN_CASES = [
+    (1024, 4, 0, 128, 128, 128, True), (32768, 8, 0, 128, 128, 128, True), (131072, 1, 8192, 128, 128, 128, True),
+    (1000, 3, 64, 128, 128, 128, True), (1, 1, 1, 1, 1, 1, True), (0, 2, 0, 8, 16, 16, True),
+    (4097, 8, 1000, 128, 64, 128, True), (300, 16, 7, 16, 32, 64, False), (8191, 5, 0, 1, 128, 128, True),
+    (127, 2, 0, 128, 128, 128, True),
+]
+
+
+@pytest.mark.parametrize("case", PLAN_CASES)
+def test_planner_matches_oracle_bit_exactly(case):
+    S, P, C, align, bm, bn, causal = case
+    tiles = S <= 40000
+    got = binding.pec_plan_partitions(S, P, C, align, bm, bn, causal, tiles=tiles)
+    want = oracle.plan_partitions(S, P, C, align, bm, bn, causal, tiles=tiles)
+    assert got["bounds"] == want["bounds"]
+    assert got["parts"] == want["parts"]
+    assert got["pairs"] == want["pairs"]
+    assert got["chunks"] == want["chunks"]
+    assert (got["nq_tiles"], got["nk_tiles"]) == (want["nq_tiles"], want["nk_tiles"])
+    if tiles:
+        assert np.array_equal(got["tile_class"], want["tile_class"])
+
+
+def test_planner_largest_config_pairs():
+    got = binding.pec_plan_partitions(262144, 16, 0, 128, 128, 128, True, tiles=False)
+    assert got["pairs"] == [8192 * 262145] * 16            # closed form b*(S+1)
+    assert got["nq_tiles"] == 2048 and got["nk_tiles"] == 2048
+
+
+def test_planner_rejects_bad_arguments_and_small_arrays():
+    lib = binding.load()
+    plan = binding.pec_plan()
+    assert lib.pec_plan_partitions(-1, 1, 0, 1, 1, 1, 1, ctypes.byref(plan)) == -1
+    assert lib.pec_plan_partitions(10, 0, 0, 1, 1, 1, 1, ctypes.byref(plan)) == -1
+    assert lib.pec_plan_partitions(10, 1, 0, 0, 1, 1, 1, ctypes.byref(plan)) == -1
+    assert lib.pec_plan_partitions(10, 1, 0, 1, 1, 1, 1, None) == -1
+    assert "plan is NULL" in binding.pec_last_error()
+    buf = (ctypes.c_int64 * 2)()
+    plan.bounds, plan.bounds_cap = buf, 2
+    assert lib.pec_plan_partitions(10, 2, 0, 1, 1, 1, 1, ctypes.byref(plan)) == -7
+    assert plan.n_bounds == 5
+
+
+def _args(**over):
+    a = binding.pec_attn_args()
+    a.q = a.k = a.v = a.o = a.lse = 4096          # never dereferenced: validation fails first
+    a.status = 4096
+    a.q_stride_t, a.q_stride_h = 8 * 128, 128
+    a.k_stride_t, a.k_stride_h = 8 * 128, 128
+    a.v_stride_t, a.v_stride_h = 8 * 128, 128
+    a.in_dtype, a.o_dtype = binding.PEC_BF16, binding.PEC_BF16
+    a.Hq, a.Hkv, a.D = 8, 8, 128
+    a.B, a.seq_len, a.chunk_start, a.chunk_len, a.kv_len = 1, 256, 0, 256, 256
+    a.part_id, a.num_parts, a.part_align, a.causal = 0, 1, 128, 1
+    for k, v in over.items():
+        setattr(a, k, v)
+    return a
+
+
+@pytest.mark.parametrize("over,code", [
+    (dict(q=None), -1), (dict(D=64), -2), (dict(Hq=6, Hkv=4), -1), (dict(in_dtype=7), -2),
+    (dict(in_dtype=binding.PEC_F32, o_dtype=binding.PEC_BF16), -2), (dict(causal=2), -1),
+    (dict(chunk_start=200, chunk_len=100), -1), (dict(kv_len=100), -1), (dict(part_id=2, num_parts=2), -1),
+    (dict(q=4100), -3), (dict(k_stride_t=8 * 128 + 4), -3), (dict(q_stride_h=64), -1),
+    (dict(cu_seqlens=4096, B=2, chunk_len=100), -1), (dict(softmax_scale=float("nan")), -1),
+    (dict(part_align=0), -1),
+])
+def test_prefill_attn_validates_on_the_host(over, code):
+    lib = binding.load()
+    a = _args(**over)
+    assert lib.pec_prefill_attn(ctypes.byref(a), None) == code
+    assert binding.pec_last_error()
+    assert lib.pec_prefill_attn(None, None) == -1
+
+
+def test_merge_validates_on_the_host():
+    lib = binding.load()
+    f = lib.pec_attn_merge
+    ok = [4096, 8192, 12288, 16384, 20480, 24576]
+    assert f(None, *ok[1:], 4, 2, 128, 2, 2, None) == -1
+    assert f(*ok, 4, 2, 64, 2, 2, None) == -2
+    assert f(*ok, 4, 2, 128, 1, 2, None) == -2
+    assert f(*ok, -1, 2, 128, 2, 2, None) == -1
+    assert f(4100, *ok[1:], 4, 2, 128, 2, 2, None) == -3
+    assert f(ok[0], ok[1], ok[2], ok[3], ok[0], ok[5], 4, 2, 128, 2, 2, None) == -1   # o aliased, lse not
+    assert f(ok[0], ok[1], ok[2], ok[3], ok[2], ok[3], 4, 2, 128, 2, 2, None) == -1   # aliasing side b
+    assert f(*ok, 0, 2, 128, 2, 2, None) == 0                                          # nothing to do
