@@ -1,0 +1,295 @@
+#!/usr/bin/env python
+"""Benchmark of the partial causal prefill attention path on B200.
+
+A step is one pass of the whole path over one synthetic long request: host plan, one partial
+attention launch per zigzag KV partition, running LSE merges, final output in the input dtype.
+Prints one JSON line (see --help for the knobs).  `--impl reference` times the fp64 CPU oracle
+on a bounded sample of the same workload instead.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2409_15104_b200 import workloads
+
+METRIC = "causal prefill attention TFLOP/s (tokens/s and % of dense BF16 peak alongside), 1 B200"
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"bf16_burst": d["bf16_tflops"], "bf16_sustained": d["bf16_tflops_sustained"],
+                "hbm": d["hbm_gbs"], "source": "measured"}
+    return {"bf16_burst": 1590.0, "bf16_sustained": 1400.0, "hbm": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(wl, q, k, v, target_s=15.0):
+    """Times the fp64 oracle, as it stands, on sampled query rows (all heads) of the workload."""
+    import oracle
+    S = wl.seq_len
+    g = np.random.Generator(np.random.Philox(key=wl.seed))
+    probe = sorted(int(x) for x in g.integers(0, S, size=4))
+    t0 = time.perf_counter()
+    oracle.prefill_attn(q, k, v, seq_len=S, rows=probe)
+    t_probe = time.perf_counter() - t0
+    n = int(max(4, min(4096, target_s / max(t_probe / len(probe), 1e-6))))
+    rows = sorted(int(x) for x in g.integers(0, S, size=n))
+    t0 = time.perf_counter()
+    oracle.prefill_attn(q, k, v, seq_len=S, rows=rows)
+    dt = time.perf_counter() - t0
+    pairs = sum(r + 1 for r in rows)
+    flops = workloads.attention_flops(pairs, wl.hq)
+    return {"seconds": dt, "rows": n, "pairs_per_head": pairs, "tflops": flops / dt / 1e12,
+            "tokens_per_s_extrapolated": S / (dt * workloads.causal_pairs(S) / pairs),
+            "cores": oracle.oracle_threads()}
+
+
+def run_reference(args, wl):
+    """--impl reference: the oracle on the host cores, each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    q, k, v = workloads.qkv(wl.seed, wl.seq_len, wl.hq, wl.hkv, 128, wl.dtype)
+    per_step = max(2.0, min(20.0, 90.0 / (args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(wl, q, k, v, target_s=per_step)
+    res = [oracle_sample(wl, q, k, v, target_s=per_step) for _ in range(args.steps)]
+    tflops = sum(r["tflops"] for r in res) / len(res)
+    ms = 1e3 * sum(r["seconds"] for r in res) / len(res)
+    sample = (f"{res[0]['rows']} seeded random query rows x all {wl.hq} heads per step, full fp64 definition per row; "
+              f"tokens/s extrapolated by pair count: {res[0]['tokens_per_s_extrapolated']:.3f}")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(wl),
+        "cpu_baseline": {"value": tflops, "unit": "TFLOP/s", "cores": res[0]["cores"], "kind": "oracle", "sample": sample},
+        "e2e": {"value": tflops, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(wl):
+    return {"workload": f"{wl.name}: {wl.note}", "seq_len": wl.seq_len, "hq": wl.hq, "hkv": wl.hkv, "head_dim": 128,
+            "num_parts": wl.num_parts, "part_align": wl.part_align, "seed": wl.seed,
+            "l2": "inputs and partials exceed the 126 MB L2; no explicit flush",
+            "flops": "4*D*Hq*(exact causal pairs), attention only, single layer"}
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def run_ours(args, wl):
+    from paper_2409_15104_b200 import binding
+    from paper_2409_15104_b200.prefill import PartitionedPrefill
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    binding.load()
+
+    # Replicas only: every rank runs the same single-GPU workload on its own seeded request.
+    seed = wl.seed + 1000 * rank
+    q_h, k_h, v_h = workloads.qkv(seed, wl.seq_len, wl.hq, wl.hkv, 128, wl.dtype)
+    q_h, k_h, v_h = q_h.pin_memory(), k_h.pin_memory(), v_h.pin_memory()
+    q, k, v = q_h.to(dev), k_h.to(dev), v_h.to(dev)
+    runner = PartitionedPrefill(wl.seq_len, wl.hq, wl.num_parts, wl.dtype, dev, wl.part_align)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        runner.run(q, k, v)
+    binding.check_status()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    runner.attn_events, runner.merge_events = [], []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for _ in range(args.steps):
+        runner.run(q, k, v, time_kernels=True)
+    t1.record(stream)
+    barrier()
+    total_ms = t0.elapsed_time(t1)
+    clocks = sampler.stop() if rank == 0 else None
+    binding.check_status()
+    attn_ms = [a.elapsed_time(b) for a, b in runner.attn_events]
+    merge_ms = [a.elapsed_time(b) for a, b in runner.merge_events]
+
+    # End to end through the public call with host buffers: H2D of Q, K, V, the path, D2H of O and LSE.
+    o_h = torch.empty((wl.seq_len, wl.hq, 128), dtype=wl.dtype).pin_memory()
+    l_h = torch.empty((wl.seq_len, wl.hq), dtype=torch.float32).pin_memory()
+    qd, kd, vd = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+
+    def e2e_step():
+        qd.copy_(q_h, non_blocking=True); kd.copy_(k_h, non_blocking=True); vd.copy_(v_h, non_blocking=True)
+        o, l = runner.run(qd, kd, vd)
+        o_h.copy_(o, non_blocking=True); l_h.copy_(l, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = max(1, min(args.steps, 5))
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    binding.check_status()
+
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(times[0]), float(times[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    pairs = workloads.causal_pairs(wl.seq_len)
+    flops_step = workloads.attention_flops(pairs, wl.hq)
+    ms_step = total_ms / args.steps
+    tflops = world * flops_step / (ms_step * 1e-3) / 1e12
+    attn_avg_ms = sum(attn_ms) / len(attn_ms)
+    flops_launch = flops_step / wl.num_parts          # zigzag partitions carry equal pair counts
+    attn_tflops = flops_launch / (attn_avg_ms * 1e-3) / 1e12
+    items = wl.seq_len * wl.hq
+    merge = None
+    if merge_ms:
+        merge_avg = sum(merge_ms) / len(merge_ms)
+        merge = {"ms_per_launch": merge_avg, "algorithmic_gbs": items * 1548 / (merge_avg * 1e-3) / 1e9,
+                 "bytes_per_item": 1548, "frac_of_measured_hbm": items * 1548 / (merge_avg * 1e-3) / 1e9 / peaks["hbm"],
+                 "frac_of_nominal_8TBs": items * 1548 / (merge_avg * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                 "note": "upper bound on bytes: rows whose side-b partial is empty are skipped by the in-place merge"}
+    h2d = q_h.numel() * q_h.element_size() + 2 * k_h.numel() * k_h.element_size()
+    d2h = o_h.numel() * o_h.element_size() + l_h.numel() * 4
+
+    cpu = oracle_sample(wl, q_h, k_h, v_h, target_s=15.0)
+    line = {
+        "metric": METRIC, "value": tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16" if wl.dtype == torch.bfloat16 else "f32", "data": "synthetic",
+        "config": workload_config(wl),
+        "tokens_per_s": world * wl.seq_len / (ms_step * 1e-3),
+        "frac_of_nominal_bf16_peak": tflops / world / NOMINAL_BF16_TFLOPS,
+        "frac_of_measured_bf16_sustained": tflops / world / peaks["bf16_sustained"],
+        "attention_only_tflops": attn_tflops,
+        "merge": merge,
+        "roofline": {"bound": "tensor", "kernel": "attn_bf16_kernel", "achieved": attn_tflops,
+                     "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": attn_tflops / peaks["bf16_sustained"],
+                     "traffic": None, "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step)",
+                     "frac_of_burst": attn_tflops / peaks["bf16_burst"], "frac_of_nominal": attn_tflops / NOMINAL_BF16_TFLOPS,
+                     "flops_per_launch": flops_launch, "ms_per_launch": attn_avg_ms},
+        "cpu_baseline": {"value": cpu["tflops"], "unit": "TFLOP/s", "cores": cpu["cores"], "kind": "oracle",
+                         "sample": f"{cpu['rows']} seeded random query rows x {wl.hq} heads of the same request, "
+                                   f"{cpu['seconds']:.1f} s; tokens/s extrapolated by pair count: "
+                                   f"{cpu['tokens_per_s_extrapolated']:.3f}"},
+        "e2e": {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": args.steps * runner.launches_per_step(),
+        "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=["c3", "c5"], default="c3")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    wl = workloads.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,124 @@
+"""The five workload configurations at full size, in the launch configuration bench.py times.
+C1 and the short requests are compared in full; the long requests on sampled rows (every head;
+rows next to every partition / chunk / tile boundary plus seeded random rows), each sampled row
+evaluated by the oracle's full definition."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import TOL, compare, sample_rows
+from paper_2409_15104_b200 import workloads
+from paper_2409_15104_b200.prefill import PartitionedPrefill, chunked_prefill, varlen_prefill
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _check_sampled(o, lse, q, k, v, S, rows, dtype, what):
+    want = oracle.prefill_attn(q, k, v, seq_len=S, rows=rows)
+    idx = torch.as_tensor(rows, device=o.device)
+    return compare(o[idx], lse[idx], *want, *TOL[dtype], what)
+
+
+def _check_varlen_sampled(o, lse, q, k, v, cu, dtype, seed, what, full_below=300, n_random=12):
+    worst = (0.0, 0.0)
+    for r in range(len(cu) - 1):
+        a, b = cu[r], cu[r + 1]
+        n = b - a
+        if n == 0:
+            continue
+        rows = list(range(n)) if n <= full_below else sample_rows(n, [128, 256, (n // 128) * 128], n_random, seed + r)
+        want = oracle.attn_rows(q[a:b][rows], np.asarray(rows), k[a:b], v[a:b], [(0, n)], True)
+        idx = torch.as_tensor(rows, device=o.device) + a
+        e = compare(o[idx], lse[idx], *want, *TOL[dtype], f"{what} request {r} (len {n})")
+        worst = (max(worst[0], e[0]), max(worst[1], e[1]))
+    return worst
+
+
+def test_c1_fp32_four_zigzag_partitions(pec):
+    wl = workloads.WORKLOADS["c1"]
+    q, k, v = workloads.qkv(wl.seed, wl.seq_len, wl.hq, wl.hkv, 128, wl.dtype)
+    plan = pec.pec_plan_partitions(wl.seq_len, wl.num_parts, 0, wl.part_align, 128, 128, True)
+    want_plan = oracle.plan_partitions(wl.seq_len, wl.num_parts, 0, wl.part_align, 128, 128, True)
+    assert plan["parts"] == want_plan["parts"] and plan["pairs"] == want_plan["pairs"]
+    assert np.array_equal(plan["tile_class"], want_plan["tile_class"])
+    runner = PartitionedPrefill(wl.seq_len, wl.hq, wl.num_parts, wl.dtype, DEV, wl.part_align)
+    o, lse = runner.run(q.to(DEV), k.to(DEV), v.to(DEV))
+    pec.check_status()
+    want = oracle.prefill_attn(q, k, v, seq_len=wl.seq_len)
+    compare(o, lse, *want, *TOL[wl.dtype], "c1")
+
+
+def test_c2_short_input_varlen_batch(pec):
+    wl = workloads.WORKLOADS["c2"]
+    lens = workloads.short_lengths(wl.seed, wl.short_batch)
+    cu = workloads.cu_seqlens(lens)
+    q, k, v = workloads.qkv(wl.seed, cu[-1], wl.hq, wl.hkv, 128, wl.dtype)
+    dcu = torch.tensor(cu, dtype=torch.int32, device=DEV)
+    o, lse = varlen_prefill(q.to(DEV), k.to(DEV), v.to(DEV), dcu)
+    pec.check_status()
+    _check_varlen_sampled(o, lse, q, k, v, cu, wl.dtype, wl.seed, "c2")
+
+
+def test_c3_long_input_eight_partitions(pec):
+    wl = workloads.WORKLOADS["c3"]
+    S = wl.seq_len
+    q, k, v = workloads.qkv(wl.seed, S, wl.hq, wl.hkv, 128, wl.dtype)
+    runner = PartitionedPrefill(S, wl.hq, wl.num_parts, wl.dtype, DEV, wl.part_align)
+    dq, dk, dv = q.to(DEV), k.to(DEV), v.to(DEV)
+    o, lse = runner.run(dq, dk, dv)
+    pec.check_status()
+    bounds = oracle.plan_partitions(S, wl.num_parts, 0, wl.part_align, 128, 128, True, tiles=False)["bounds"]
+    rows = sample_rows(S, bounds + [127, 128, 129], 256, wl.seed)
+    _check_sampled(o, lse, q, k, v, S, rows, wl.dtype, "c3 merged")
+    # one partial at full size: partition 3 on a smaller sample
+    po, pl = pec.pec_prefill_attn(dq, dk, dv, part_id=3, num_parts=wl.num_parts, part_align=wl.part_align)
+    pec.check_status()
+    prow = sample_rows(S, bounds, 24, wl.seed + 1)
+    want = oracle.prefill_attn(q, k, v, seq_len=S, part_id=3, num_parts=wl.num_parts, part_align=wl.part_align, rows=prow)
+    idx = torch.as_tensor(prow, device=DEV)
+    compare(po[idx], pl[idx], *want, *TOL[wl.dtype], "c3 partition 3")
+
+
+def test_c4_preempted_chunks_with_colocated_short_batch(pec):
+    wl = workloads.WORKLOADS["c4"]
+    S, C = wl.seq_len, wl.chunk_len
+    q, k, v = workloads.qkv(wl.seed, S, wl.hq, wl.hkv, 128, wl.dtype)
+    lens = workloads.short_lengths(wl.seed, wl.short_batch)
+    cu = workloads.cu_seqlens(lens)
+    sq, sk, sv = workloads.qkv(wl.seed + 100, cu[-1], wl.hq, wl.hkv, 128, wl.dtype)
+    dq, dk, dv = q.to(DEV), k.to(DEV), v.to(DEV)
+    dsq, dsk, dsv = sq.to(DEV), sk.to(DEV), sv.to(DEV)
+    dcu = torch.tensor(cu, dtype=torch.int32, device=DEV)
+    o = torch.empty((S, wl.hq, 128), dtype=wl.dtype, device=DEV)
+    lse = torch.empty((S, wl.hq), dtype=torch.float32, device=DEV)
+    so = torch.empty((cu[-1], wl.hq, 128), dtype=wl.dtype, device=DEV)
+    sl = torch.empty((cu[-1], wl.hq), dtype=torch.float32, device=DEV)
+    lo_prio, hi_prio = torch.cuda.Stream(priority=0), torch.cuda.Stream(priority=-1)
+    torch.cuda.synchronize()
+
+    def preempt(c):          # the short batch arrives after chunks 3 and 9 have been enqueued
+        if c in (3, 9):
+            varlen_prefill(dsq, dsk, dsv, dcu, o=so, lse=sl, stream=hi_prio)
+
+    chunks = chunked_prefill(dq, dk, dv, C, o, lse, stream=lo_prio, between_chunks=preempt)
+    torch.cuda.synchronize()
+    pec.check_status()
+    assert len(chunks) == 16
+    bounds = [c0 for c0, _ in chunks] + [S]
+    rows = sample_rows(S, bounds, 160, wl.seed)
+    _check_sampled(o, lse, q, k, v, S, rows, wl.dtype, "c4 long request")
+    _check_varlen_sampled(so, sl, sq, sk, sv, cu, wl.dtype, wl.seed, "c4 short batch", full_below=130, n_random=6)
+
+
+def test_c5_very_long_input_sixteen_partitions(pec):
+    wl = workloads.WORKLOADS["c5"]
+    S = wl.seq_len
+    q, k, v = workloads.qkv(wl.seed, S, wl.hq, wl.hkv, 128, wl.dtype)
+    runner = PartitionedPrefill(S, wl.hq, wl.num_parts, wl.dtype, DEV, wl.part_align)
+    o, lse = runner.run(q.to(DEV), k.to(DEV), v.to(DEV))
+    pec.check_status()
+    bounds = oracle.plan_partitions(S, wl.num_parts, 0, wl.part_align, 128, 128, True, tiles=False)["bounds"]
+    rows = sample_rows(S, bounds[::4], 96, wl.seed)
+    _check_sampled(o, lse, q, k, v, S, rows, wl.dtype, "c5 merged")
