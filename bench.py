@@ -193,6 +193,17 @@ def run_ours(args, wl):
     attn_ms = [a.elapsed_time(b) for a, b in runner.attn_events]
     merge_ms = [a.elapsed_time(b) for a, b in runner.merge_events]
 
+    if args.profile:
+        if rank == 0:
+            fl = workloads.attention_flops(workloads.causal_pairs(wl.seq_len), wl.hq)
+            print(json.dumps({"profile_run": True, "ms_per_step": total_ms / args.steps,
+                              "attn_ms_per_launch": sum(attn_ms) / len(attn_ms),
+                              "attn_tflops": fl / wl.num_parts / (sum(attn_ms) / len(attn_ms)) / 1e9,
+                              "merge_ms_per_launch": (sum(merge_ms) / len(merge_ms)) if merge_ms else None}), flush=True)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
     # End to end through the public call with host buffers: H2D of Q, K, V, the path, D2H of O and LSE.
     o_h = torch.empty((wl.seq_len, wl.hq, 128), dtype=wl.dtype).pin_memory()
     l_h = torch.empty((wl.seq_len, wl.hq), dtype=torch.float32).pin_memory()
@@ -276,10 +287,12 @@ def run_ours(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=["c3", "c5"], default="c3")
+    ap.add_argument("--profile", action="store_true",
+                    help="profiling runs: skip the end-to-end and CPU-baseline legs (the printed line is not a result)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = workloads.WORKLOADS[args.workload]

@@ -1,12 +1,22 @@
 // bf16 partial causal attention on the sm_100a tensor cores (Eq. 3-4 as KV-tile partial attention
 // with online-softmax state: running max, running sum, fp32 accumulator).
 //
-// One CTA = one (128-row query tile, head).  Q, K and V tiles arrive by TMA into 128-byte-swizzled
-// shared memory; S = Q K^T and O += P V run as tcgen05.mma with fp32 accumulators in tensor
-// memory (TMEM); the four warps own the 128 TMEM lanes (one query row per thread) for the softmax.
-// P is written back to TMEM as packed bf16 and consumed as the A operand of the second MMA.
+// One CTA = one head x 256 query rows, handled as two 128-row tiles ("stages") that ping-pong on
+// the tensor core.  Warp roles:
+//   warps 0-3  softmax of stage 0 (one query row per thread = one TMEM lane)
+//   warps 4-7  softmax of stage 1
+//   warp  8    MMA issuer (one elected lane issues every tcgen05.mma)
+//   warp  9    TMA loader (Q once, then K and V tiles through a ring of shared-memory slots)
+//   warps 10-11 idle; they complete the third warpgroup so that it can hand its registers to the
+//              softmax warpgroups (setmaxnreg acts on whole warpgroups)
+// S = Q K^T lands in tensor memory, the softmax warps turn it into P (bf16, written back over the
+// first half of S), and O += P V accumulates in tensor memory; the issue order
+//   PV_0(j), S_0(j+1), PV_1(j), S_1(j+1), ...
+// lets one stage's softmax run under the other stage's two MMAs.  The accumulator is rescaled
+// lazily: the reference maximum of a row only moves when the new maximum exceeds it by 2^8.
 //
-// TMEM columns: [0,128) S (fp32), reused as P (bf16 pairs, columns [0,64)); [128,256) O (fp32).
+// TMEM columns: S_0 [0,128) (P_0 in [0,64)), S_1 [128,256) (P_1 in [128,192)), O_0 [256,384),
+// O_1 [384,512).
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -17,20 +27,28 @@
 namespace pec {
 using namespace sm100;
 
-constexpr int kTileM = 128, kTileN = 128;
-constexpr int kThreads = 128;
+constexpr int kTile = 128;                                 // rows per stage, keys per KV tile
+constexpr int kBlockM = 2 * kTile;                         // query rows per CTA
+constexpr int kStages = 4;                                 // K/V ring slots
+constexpr int kThreads = 384;                              // three full warpgroups (setmaxnreg is per warpgroup)
+constexpr int kMmaWarp = 8, kLoadWarp = 9;
+constexpr int kLightRegs = 56, kSoftmaxRegs = 224;          // per sub-partition: 2 * 224 + 56 <= 512
 constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;          // one TMA box: 128 rows x 64 bf16
 constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;        // 128 x 128 bf16
-constexpr uint32_t kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColP = 0, kColO = 128;
-constexpr size_t kSmemBytes = 3 * kTileBytes + 1024 /*alignment slack*/ + 64 /*barriers*/;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256;                 // + 128 * stage
+constexpr float kRescaleThreshold = 8.0f;                  // log2 units
+constexpr int kPolyOf4 = 0;                                // pairs of every 4 whose 2^x runs on the FMA pipe
 constexpr long long kWaitCycles = 2000000000LL;            // bounded waits give up after ~1 s
 
 struct Shared {
-    uint64_t bar_q, bar_kv, bar_mma;
+    uint64_t bar_q;
+    uint64_t kv_full[kStages], kv_empty[kStages];
+    uint64_t s_full[2], p_ready[2], o_final[2];
     uint32_t tmem_base;
     volatile int abort_flag;
 };
+constexpr size_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*alignment slack*/ + sizeof(Shared);
 
 // Bounded mbarrier wait.  Returns false (and raises the abort flag / status word) on expiry.
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *sh, int32_t *status)
@@ -48,6 +66,17 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *
     return true;
 }
 
+// Key tiles a CTA walks: the tiles of interval 0, then those of interval 1, in ascending position.
+struct TileWalk {
+    int64_t lo[2], hi[2];
+    int32_t cnt[2];          // tiles per interval for the CTA (union over both stages)
+    __device__ __forceinline__ void at(int j, int64_t &k0, int64_t &hi_t) const
+    {
+        if (j < cnt[0]) { k0 = lo[0] + (int64_t)j * kTile; hi_t = hi[0]; }
+        else            { k0 = lo[1] + (int64_t)(j - cnt[0]) * kTile; hi_t = hi[1]; }
+    }
+};
+
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const AttnParams p)
@@ -55,16 +84,15 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
-    const uint32_t sQ = tiles, sK = tiles + kTileBytes, sV = tiles + 2 * kTileBytes;
-    Shared *sh = reinterpret_cast<Shared *>(smem_raw + (tiles - raw) + 3 * kTileBytes);
-    const uint32_t bar_q = smem_u32(&sh->bar_q), bar_kv = smem_u32(&sh->bar_kv), bar_mma = smem_u32(&sh->bar_mma);
+    const uint32_t sQ = tiles, sRing = tiles + 2 * kTileBytes;
+    Shared *sh = reinterpret_cast<Shared *>(smem_raw + (tiles - raw) + (2 + kStages) * kTileBytes);
 
     // Heaviest (latest) causal tiles first.
     const int64_t tile = (int64_t)gridDim.x - 1 - blockIdx.x;
     TileJob job;
-    if (!locate_tile(p, tile, kTileM, job)) return;
+    if (!locate_tile(p, tile, kBlockM, job)) return;
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.y, kvh = h / p.group;
 
     // An earlier CTA's wait expired: the launch is already lost, leave at once (uniform decision).
@@ -72,10 +100,39 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     __syncthreads();
     if (sh->abort_flag) return;
 
+    // Per-stage geometry: rows, positions and how many key tiles each stage takes part in.
+    int32_t rows_st[2], n_st[2];
+    int64_t pos0_st[2];
+    TileWalk walk;
+    walk.cnt[0] = walk.cnt[1] = 0;
+    for (int t = 0; t < 2; ++t) { walk.lo[t] = job.iv_lo[t]; walk.hi[t] = job.iv_hi[t]; }
+#pragma unroll
+    for (int st = 0; st < 2; ++st) {
+        rows_st[st] = job.n_rows - st * kTile;
+        rows_st[st] = rows_st[st] < 0 ? 0 : (rows_st[st] > kTile ? kTile : rows_st[st]);
+        pos0_st[st] = job.q_pos0 + st * kTile;
+        n_st[st] = 0;
+        if (rows_st[st] > 0) {
+            const int64_t last = pos0_st[st] + rows_st[st] - 1;
+            for (int t = 0; t < job.n_iv; ++t) {
+                int64_t end = job.iv_hi[t];
+                if (p.causal && end > last + 1) end = last + 1;
+                const int32_t c = end > job.iv_lo[t] ? (int32_t)((end - job.iv_lo[t] + kTile - 1) / kTile) : 0;
+                n_st[st] += c;
+                walk.cnt[t] = c > walk.cnt[t] ? c : walk.cnt[t];
+            }
+        }
+    }
+    const int n_max = walk.cnt[0] + walk.cnt[1];
+
     if (tid == 0) {
-        mbar_init(bar_q, 1);
-        mbar_init(bar_kv, 1);
-        mbar_init(bar_mma, 1);
+        mbar_init(smem_u32(&sh->bar_q), 1);
+        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->kv_full[s]), 1); mbar_init(smem_u32(&sh->kv_empty[s]), 1); }
+        for (int st = 0; st < 2; ++st) {
+            mbar_init(smem_u32(&sh->s_full[st]), 1);
+            mbar_init(smem_u32(&sh->p_ready[st]), 4);         // one arrival per softmax warp
+            mbar_init(smem_u32(&sh->o_final[st]), 1);
+        }
         mbar_init_fence();
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
     }
@@ -88,166 +145,236 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sh->tmem_base;
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;  // this warp's TMEM lanes
 
-    if (tid == 0) {
-        mbar_arrive_expect_tx(bar_q, kTileBytes);
-        tma_load_3d(sQ, &tm_q, bar_q, 0, h, (int)job.q_row0);
-        tma_load_3d(sQ + kHalfTileBytes, &tm_q, bar_q, 64, h, (int)job.q_row0);
-    }
-
-    constexpr uint32_t idesc_qk = idesc_bf16_f32(kTileM, kTileN, 0, 0);
-    constexpr uint32_t idesc_pv = idesc_bf16_f32(kTileM, kHeadDim, 0, 1);
-
-    float m_run = -INFINITY, l_run = 0.f;
-    const int64_t my_pos = job.q_pos0 + tid;
-    const int64_t last_pos = job.q_pos0 + job.n_rows - 1;
-    uint32_t kv_phase = 0, mma_phase = 0;
-    bool first = true, ok = true;
-
-    for (int t = 0; t < job.n_iv && ok; ++t) {
-        const int64_t lo = job.iv_lo[t];
-        const int64_t hi = job.iv_hi[t];
-        int64_t end = hi;                                     // keys at or after `end` are invisible to the whole tile
-        if (p.causal && end > last_pos + 1) end = last_pos + 1;
-        for (int64_t k0 = lo; k0 < end && ok; k0 += kTileN) {
-            if (tid == 0) {
-                const int krow = (int)(job.kv_row0 + k0);
-                mbar_arrive_expect_tx(bar_kv, 2 * kTileBytes);
-                tma_load_3d(sK, &tm_k, bar_kv, 0, kvh, krow);
-                tma_load_3d(sK + kHalfTileBytes, &tm_k, bar_kv, 64, kvh, krow);
-                tma_load_3d(sV, &tm_v, bar_kv, 0, kvh, krow);
-                tma_load_3d(sV + kHalfTileBytes, &tm_v, bar_kv, 64, kvh, krow);
-                if (first) ok = wait_bar(bar_q, 0, sh, p.status);
-                ok = ok && wait_bar(bar_kv, kv_phase, sh, p.status);
-                if (ok) {
-                    // S = Q K^T: both operands K-major; 8 steps of 16 channels, 4 per 64-channel half tile
+    // Warps 8-11 (the whole third warpgroup) give registers up, warps 0-7 take them.
+    if (warp == kLoadWarp) {
+        // ------------------------------------------------------------------ TMA loader
+        reg_dealloc<kLightRegs>();
+        if (lane == 0 && n_max > 0) {
+            const uint32_t bar_q = smem_u32(&sh->bar_q);
+            mbar_arrive_expect_tx(bar_q, 2 * kTileBytes);
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint32_t off = (uint32_t)(ks >> 2) * kHalfTileBytes + (uint32_t)(ks & 3) * 32u;
-                        mma_ss(tmem + kColS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024),
-                               idesc_qk, ks > 0 ? 1u : 0u);
-                    }
-                    tc_commit(bar_mma);
-                }
+            for (int st = 0; st < 2; ++st) {
+                const int row = (int)(job.q_row0 + st * kTile);
+                tma_load_3d(sQ + st * kTileBytes, &tm_q, bar_q, 0, h, row);
+                tma_load_3d(sQ + st * kTileBytes + kHalfTileBytes, &tm_q, bar_q, 64, h, row);
             }
-            kv_phase ^= 1;
-            ok = __all_sync(0xffffffffu, wait_bar(bar_mma, mma_phase, sh, p.status));   // warp-uniform
-            mma_phase ^= 1;
+            for (int i = 0; i < 2 * n_max; ++i) {              // items: K(0), V(0), K(1), V(1), ...
+                const int slot = i % kStages, fill = i / kStages;
+                if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p.status)) break;
+                int64_t k0, hi_t;
+                walk.at(i >> 1, k0, hi_t);
+                const int krow = (int)(job.kv_row0 + k0);
+                const uint32_t dst = sRing + slot * kTileBytes, bar = smem_u32(&sh->kv_full[slot]);
+                const void *map = (i & 1) ? (const void *)&tm_v : (const void *)&tm_k;
+                mbar_arrive_expect_tx(bar, kTileBytes);
+                tma_load_3d(dst, map, bar, 0, kvh, krow);
+                tma_load_3d(dst + kHalfTileBytes, map, bar, 64, kvh, krow);
+            }
+        }
+        __syncwarp();
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issuer
+        reg_dealloc<kLightRegs>();
+        if (lane == 0 && n_max > 0) {
+            constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kTile, 0, 0);
+            constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, kHeadDim, 0, 1);
+            auto kv_wait = [&](int item) {
+                return wait_bar(smem_u32(&sh->kv_full[item % kStages]), (item / kStages) & 1, sh, p.status);
+            };
+            auto kv_release = [&](int item) { tc_commit(smem_u32(&sh->kv_empty[item % kStages])); };
+            // S_st = Q_st K^T: both operands K-major; 8 steps of 16 channels, 4 per 64-channel half tile
+            auto issue_qk = [&](int st, int item) {
+                const uint32_t a = sQ + st * kTileBytes, b = sRing + (item % kStages) * kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (uint32_t)(ks >> 2) * kHalfTileBytes + (uint32_t)(ks & 3) * 32u;
+                    mma_ss(tmem + kColS + st * kTile, smem_desc_sw128(a + off, 16, 1024), smem_desc_sw128(b + off, 16, 1024),
+                           idesc_qk, ks > 0 ? 1u : 0u);
+                }
+                tc_commit(smem_u32(&sh->s_full[st]));
+            };
+            // O_st (+)= P_st V: A = P from TMEM (8 columns per 16 keys), B = V tile stored [key][channel]
+            // (N-contiguous): 16 keys = 2048 bytes per step, channel halves 16 KiB apart.
+            auto issue_pv = [&](int st, int item, bool accumulate) {
+                const uint32_t b = sRing + (item % kStages) * kTileBytes;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks)
+                    mma_ts(tmem + kColO + st * kTile, tmem + kColS + st * kTile + ks * 8,
+                           smem_desc_sw128(b + ks * 2048u, kHalfTileBytes, 1024), idesc_pv, (accumulate || ks > 0) ? 1u : 0u);
+            };
+
+            bool ok = wait_bar(smem_u32(&sh->bar_q), 0, sh, p.status) && kv_wait(0);
+            if (ok) {
+                if (n_st[0] > 0) issue_qk(0, 0);
+                if (n_st[1] > 0) issue_qk(1, 0);
+                kv_release(0);
+            }
+            for (int j = 0; j < n_max && ok; ++j) {
+                const bool has_next = j + 1 < n_max;
+                ok = kv_wait(2 * j + 1);                       // V(j)
+#pragma unroll
+                for (int st = 0; st < 2 && ok; ++st) {
+                    if (j < n_st[st]) {
+                        ok = wait_bar(smem_u32(&sh->p_ready[st]), j & 1, sh, p.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(st, 2 * j + 1, j > 0);
+                        if (j == n_st[st] - 1) tc_commit(smem_u32(&sh->o_final[st]));
+                    }
+                    if (st == 0 && has_next) { ok = kv_wait(2 * j + 2); if (!ok) break; }   // K(j+1)
+                    if (j + 1 < n_st[st]) issue_qk(st, 2 * j + 2);
+                }
+                if (!ok) break;
+                kv_release(2 * j + 1);
+                if (has_next) kv_release(2 * j + 2);
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 8) {
+        reg_dealloc<kLightRegs>();
+    } else {
+        // ------------------------------------------------------------------ softmax + epilogue
+        reg_alloc<kSoftmaxRegs>();
+        const int st = warp >> 2;
+        const int row_in_tile = (warp & 3) * 32 + lane;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_base + kColS + st * kTile;
+        const uint32_t tO = tmem + lane_base + kColO + st * kTile;
+        const int64_t my_pos = pos0_st[st] + row_in_tile;
+        const int n_mine = n_st[st];
+        const uint32_t bar_s = smem_u32(&sh->s_full[st]), bar_p = smem_u32(&sh->p_ready[st]);
+
+        float m_ref = -INFINITY, l_run = 0.f;                // m_ref in log2 units of the scaled scores
+        bool ok = true;
+        for (int j = 0; j < n_mine; ++j) {
+            ok = __all_sync(0xffffffffu, wait_bar(bar_s, j & 1, sh, p.status));     // warp-uniform
             if (!ok) break;
             tc_fence_after();
 
-            // visible columns of this row inside the tile
-            int64_t lim = hi;
-            if (p.causal && my_pos + 1 < lim) lim = my_pos + 1;
-            int n_vis = (int)(lim - k0);
-            n_vis = n_vis < 0 ? 0 : (n_vis > kTileN ? kTileN : n_vis);
-
-            float s[kTileN];
+            uint32_t r[kTile];
+            tmem_ld128(tS, r);
+            int64_t k0, hi_t;
+            walk.at(j, k0, hi_t);
+            // Mask only when some row of this stage cannot see the whole tile.
+            int64_t full_lim = hi_t;
+            if (p.causal && pos0_st[st] + 1 < full_lim) full_lim = pos0_st[st] + 1;
+            const bool masked = k0 + kTile > full_lim;
+            if (masked) {
+                int64_t lim = hi_t;
+                if (p.causal && my_pos + 1 < lim) lim = my_pos + 1;
+                int n_vis = (int)(lim - k0);
+                n_vis = n_vis < 0 ? 0 : (n_vis > kTile ? kTile : n_vis);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tmem + lane_base + kColS + c * 32, r);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) s[c * 32 + j] = __uint_as_float(r[j]);
+                for (int c = 0; c < kTile; ++c) r[c] = (c < n_vis) ? r[c] : 0xff800000u;   // -inf
             }
-            float mx = -INFINITY;
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < kTileN; ++j) {
-                s[j] = (j < n_vis) ? s[j] * p.scale_log2 : -INFINITY;
-                mx = fmaxf(mx, s[j]);
+            for (int c = 0; c < kTile; c += 8) {
+                mx0 = fmax3(mx0, __uint_as_float(r[c + 0]), __uint_as_float(r[c + 1]));
+                mx1 = fmax3(mx1, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+                mx2 = fmax3(mx2, __uint_as_float(r[c + 4]), __uint_as_float(r[c + 5]));
+                mx3 = fmax3(mx3, __uint_as_float(r[c + 6]), __uint_as_float(r[c + 7]));
             }
-            const float m_new = fmaxf(m_run, mx);
-            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
-            const float alpha = ex2(m_run - m_use);           // 0 while the row has seen no key
-            float rs = 0.f;
-#pragma unroll
-            for (int j = 0; j < kTileN; ++j) { s[j] = ex2(s[j] - m_use); rs += s[j]; }
-            l_run = l_run * alpha + rs;
-            m_run = m_new;
+            const float m_new = fmax3(mx0, mx1, fmaxf(mx2, mx3)) * p.scale_log2;   // -inf stays -inf (scale > 0)
 
-            if (!first) {                                     // rescale the accumulator rows
+            // Lazy rescale: move the reference maximum only when it is outgrown by 2^8.
+            float alpha = 1.f;
+            const bool grow = m_new > m_ref + kRescaleThreshold;
+            if (grow) {
+                alpha = ex2(m_ref - m_new);                   // 0 when the row had no key so far
+                m_ref = m_new;
+                l_run *= alpha;
+            }
+            if (j > 0 && __any_sync(0xffffffffu, grow)) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(tmem + lane_base + kColO + c * 32, r);
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
-                    tmem_st32(tmem + lane_base + kColO + c * 32, r);
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st32(tO + c * 32, o);
                 }
             }
-            // P as packed bf16: column c of the A operand holds keys 2c (low half) and 2c+1 (high half)
+            const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(neg_m, neg_m);
+            float2 sum[4];
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t r[32];
+            for (int i = 0; i < 4; ++i) sum[i] = make_float2(0.f, 0.f);
+            // p = 2^(s * scale - m): packed FMA for the argument, then the special-function unit, or for
+            // kPolyOf4 of every 4 pairs of an unmasked tile, the FMA/integer pipes.  P is packed to bf16
+            // pairs: column c of the A operand holds keys 2c (low half) and 2c+1 (high half).
+            if (masked) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = pack_bf16(s[c * 64 + 2 * j], s[c * 64 + 2 * j + 1]);
-                tmem_st32(tmem + lane_base + kColP + c * 32, r);
+                for (int i = 0; i < kTile / 2; ++i) {
+                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, nm2);
+                    const float2 e = make_float2(ex2(x.x), ex2(x.y));
+                    sum[i & 3] = __fadd2_rn(sum[i & 3], e);
+                    r[i] = pack_bf16(e.x, e.y);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < kTile / 2; ++i) {
+                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, nm2);
+                    const float2 e = ((i & 3) < kPolyOf4) ? ex2_poly2(x) : make_float2(ex2(x.x), ex2(x.y));
+                    sum[i & 3] = __fadd2_rn(sum[i & 3], e);
+                    r[i] = pack_bf16(e.x, e.y);
+                }
+            }
+            const float2 s01 = __fadd2_rn(__fadd2_rn(sum[0], sum[1]), __fadd2_rn(sum[2], sum[3]));
+            l_run += s01.x + s01.y;
+            {
+                uint32_t(&lo)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[0]);
+                uint32_t(&hi)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[32]);
+                tmem_st32(tS, lo);
+                tmem_st32(tS + 32, hi);
             }
             tmem_st_wait();
             tc_fence_before();
-            __syncthreads();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_p);
+        }
 
-            if (tid == 0) {
-                tc_fence_after();
-                // O (+)= P V: A = P from TMEM (8 columns per 16 keys), B = V tile stored [key][channel]
-                // (N-contiguous): 16 keys = 2048 bytes per step, channel halves 16 KiB apart.
-#pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    mma_ts(tmem + kColO, tmem + kColP + ks * 8, smem_desc_sw128(sV + ks * 2048u, kHalfTileBytes, 1024),
-                           idesc_pv, (!first || ks > 0) ? 1u : 0u);
-                }
-                tc_commit(bar_mma);
-            }
-            ok = __all_sync(0xffffffffu, wait_bar(bar_mma, mma_phase, sh, p.status));
-            mma_phase ^= 1;
+        // Epilogue: O / l and LSE = ln2 * m + ln l; rows without any visible key give 0 and -inf.
+        if (ok && n_mine > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->o_final[st]), 0, sh, p.status));
+        if (ok && rows_st[st] > 0) {
             tc_fence_after();
-            first = false;
-        }
-    }
-
-    // A tile without any key tile never consumed its Q copy: let it land before the CTA retires.
-    if (first && tid == 0) wait_bar(bar_q, 0, sh, p.status);
-    __syncwarp();
-
-    // Epilogue: O / l and LSE = ln2 * m + ln l; rows without any visible key give 0 and -inf.
-    // (TMEM loads are warp-wide; only the global stores are predicated on the row being valid.)
-    if (ok) {
-        const bool valid = tid < job.n_rows;
-        const bool empty = (l_run == 0.f);
-        const float inv = empty ? 0.f : 1.f / l_run;
-        const int64_t row = job.out_row0 + tid;
-        const int64_t obase = (row * p.Hq + h) * kHeadDim;
+            const bool valid = row_in_tile < rows_st[st];
+            const bool empty = (l_run == 0.f);
+            const float inv = empty ? 0.f : 1.f / l_run;
+            const int64_t row = job.out_row0 + st * kTile + row_in_tile;
+            const int64_t obase = (row * p.Hq + h) * kHeadDim;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            uint32_t r[32];
-            if (first) {
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                if (n_mine == 0) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = 0u;
-            } else {
-                tmem_ld32(tmem + lane_base + kColO + c * 32, r);
-            }
-            if (!valid) continue;
-            if (p.o_is_bf16) {
-                __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(p.o) + obase + c * 32;
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                    uint4 pk;
-                    pk.x = pack_bf16(__uint_as_float(r[j + 0]) * inv, __uint_as_float(r[j + 1]) * inv);
-                    pk.y = pack_bf16(__uint_as_float(r[j + 2]) * inv, __uint_as_float(r[j + 3]) * inv);
-                    pk.z = pack_bf16(__uint_as_float(r[j + 4]) * inv, __uint_as_float(r[j + 5]) * inv);
-                    pk.w = pack_bf16(__uint_as_float(r[j + 6]) * inv, __uint_as_float(r[j + 7]) * inv);
-                    *reinterpret_cast<uint4 *>(o + j) = pk;
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;
+                } else {
+                    tmem_ld32(tO + c * 32, r);                // warp-wide; only the stores are predicated
                 }
-            } else {
-                float *o = static_cast<float *>(p.o) + obase + c * 32;
+                if (!valid) continue;
+                if (p.o_is_bf16) {
+                    __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(p.o) + obase + c * 32;
 #pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                    *reinterpret_cast<float4 *>(o + j) = make_float4(__uint_as_float(r[j]) * inv, __uint_as_float(r[j + 1]) * inv,
-                                                                     __uint_as_float(r[j + 2]) * inv, __uint_as_float(r[j + 3]) * inv);
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 pk;
+                        pk.x = pack_bf16(__uint_as_float(r[i + 0]) * inv, __uint_as_float(r[i + 1]) * inv);
+                        pk.y = pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+                        pk.z = pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
+                        pk.w = pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(o + i) = pk;
+                    }
+                } else {
+                    float *o = static_cast<float *>(p.o) + obase + c * 32;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        *reinterpret_cast<float4 *>(o + i) = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
+                                                                         __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+                }
             }
+            if (valid) p.lse[row * p.Hq + h] = empty ? -INFINITY : m_ref * 0.6931471805599453f + logf(l_run);
         }
-        if (valid) p.lse[row * p.Hq + h] = empty ? -INFINITY : m_run * 0.6931471805599453f + logf(l_run);
     }
 
     tc_fence_before();
@@ -309,7 +436,7 @@ int launch_attn_bf16(const AttnParams &p, cudaStream_t stream)
         set_error("pec_prefill_attn: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
         return PEC_ERR_CUDA;
     }
-    int64_t tiles = (p.total_rows + kTileM - 1) / kTileM;
+    int64_t tiles = (p.total_rows + kBlockM - 1) / kBlockM;
     if (p.cu_seqlens) tiles += p.B;
     if (tiles > 0x7fffffff || p.Hq > 65535) { set_error("pec_prefill_attn: grid too large"); return PEC_ERR_UNSUPPORTED; }
     dim3 grid((unsigned)tiles, (unsigned)p.Hq);
