@@ -2,13 +2,13 @@
 // with online-softmax state: running max, running sum, fp32 accumulator).
 //
 // One CTA = one head x 256 query rows, handled as two 128-row tiles ("stages") that ping-pong on
-// the tensor core.  Warp roles:
-//   warps 0-3  softmax of stage 0 (one query row per thread = one TMEM lane)
-//   warps 4-7  softmax of stage 1
-//   warp  8    MMA issuer (one elected lane issues every tcgen05.mma)
-//   warp  9    TMA loader (Q once, then K and V tiles through a ring of shared-memory slots)
+// the tensor core.  Warp roles (three warpgroups):
+//   warps 0-3   softmax of stage 0 (one query row per thread = one TMEM lane)
+//   warps 4-7   softmax of stage 1
+//   warp  8     MMA issuer (one elected lane issues every tcgen05.mma)
+//   warp  9     TMA loader (Q once, then K and V tiles through a ring of shared-memory slots)
 //   warps 10-11 idle; they complete the third warpgroup so that it can hand its registers to the
-//              softmax warpgroups (setmaxnreg acts on whole warpgroups)
+//               softmax warpgroups (setmaxnreg acts on whole warpgroups)
 // S = Q K^T lands in tensor memory, the softmax warps turn it into P (bf16, written back over the
 // first half of S), and O += P V accumulates in tensor memory; the issue order
 //   PV_0(j), S_0(j+1), PV_1(j), S_1(j+1), ...
@@ -30,9 +30,9 @@ using namespace sm100;
 constexpr int kTile = 128;                                 // rows per stage, keys per KV tile
 constexpr int kBlockM = 2 * kTile;                         // query rows per CTA
 constexpr int kStages = 4;                                 // K/V ring slots
-constexpr int kThreads = 384;                              // three full warpgroups (setmaxnreg is per warpgroup)
-constexpr int kMmaWarp = 8, kLoadWarp = 9;
-constexpr int kLightRegs = 56, kSoftmaxRegs = 224;          // per sub-partition: 2 * 224 + 56 <= 512
+constexpr int kThreads = 384;                              // three full warpgroups
+constexpr int kSoftmaxWarps = 8, kMmaWarp = 8, kLoadWarp = 9;
+constexpr int kLightRegs = 56, kSoftmaxRegs = 224;          // 256 * 224 + 128 * 56 = 384 * 168 (the launch allocation)
 constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;          // one TMA box: 128 rows x 64 bf16
 constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;        // 128 x 128 bf16
 constexpr uint32_t kTmemCols = 512;
@@ -40,11 +40,26 @@ constexpr uint32_t kColS = 0, kColO = 256;                 // + 128 * stage
 constexpr float kRescaleThreshold = 8.0f;                  // log2 units
 constexpr int kPolyOf4 = 0;                                // pairs of every 4 whose 2^x runs on the FMA pipe
 constexpr long long kWaitCycles = 2000000000LL;            // bounded waits give up after ~1 s
+constexpr uint32_t kSuspendNs = 2000;                      // a waiting thread sleeps in the barrier unit this long per try
+
+// What a CTA works on, worked out once by thread 0 and shared through shared memory.  All rows and
+// positions fit in 32 bits (the host rejects larger problems).
+struct Geom {
+    int32_t found;               // 0: tile index past the end (or the launch was already aborted)
+    int32_t q_row0, out_row0, kv_row0;
+    int32_t rows[2];             // valid query rows per stage
+    int32_t pos0[2];             // position of each stage's first row in its request
+    int32_t n[2];                // key tiles each stage takes part in (a prefix of the CTA's walk)
+    int32_t lo[2], hi[2];        // visible-key intervals (positions)
+    int32_t cnt[2];              // key tiles per interval walked by the CTA (union over both stages)
+    int32_t n_max;               // cnt[0] + cnt[1]
+};
 
 struct Shared {
     uint64_t bar_q;
     uint64_t kv_full[kStages], kv_empty[kStages];
     uint64_t s_full[2], p_ready[2], o_final[2];
+    Geom g;
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -55,7 +70,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
+    while (!mbar_try_wait_suspend(bar, parity, kSuspendNs)) {
         if (sh->abort_flag) return false;
         if (clock64() - t0 > kWaitCycles) {
             sh->abort_flag = 1;
@@ -65,17 +80,6 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *
     }
     return true;
 }
-
-// Key tiles a CTA walks: the tiles of interval 0, then those of interval 1, in ascending position.
-struct TileWalk {
-    int64_t lo[2], hi[2];
-    int32_t cnt[2];          // tiles per interval for the CTA (union over both stages)
-    __device__ __forceinline__ void at(int j, int64_t &k0, int64_t &hi_t) const
-    {
-        if (j < cnt[0]) { k0 = lo[0] + (int64_t)j * kTile; hi_t = hi[0]; }
-        else            { k0 = lo[1] + (int64_t)(j - cnt[0]) * kTile; hi_t = hi[1]; }
-    }
-};
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -87,43 +91,47 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const uint32_t sQ = tiles, sRing = tiles + 2 * kTileBytes;
     Shared *sh = reinterpret_cast<Shared *>(smem_raw + (tiles - raw) + (2 + kStages) * kTileBytes);
 
-    // Heaviest (latest) causal tiles first.
-    const int64_t tile = (int64_t)gridDim.x - 1 - blockIdx.x;
-    TileJob job;
-    if (!locate_tile(p, tile, kBlockM, job)) return;
-
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.y, kvh = h / p.group;
 
-    // An earlier CTA's wait expired: the launch is already lost, leave at once (uniform decision).
-    if (tid == 0) sh->abort_flag = (p.status && *reinterpret_cast<volatile int32_t *>(p.status) != 0) ? 1 : 0;
-    __syncthreads();
-    if (sh->abort_flag) return;
-
-    // Per-stage geometry: rows, positions and how many key tiles each stage takes part in.
-    int32_t rows_st[2], n_st[2];
-    int64_t pos0_st[2];
-    TileWalk walk;
-    walk.cnt[0] = walk.cnt[1] = 0;
-    for (int t = 0; t < 2; ++t) { walk.lo[t] = job.iv_lo[t]; walk.hi[t] = job.iv_hi[t]; }
-#pragma unroll
-    for (int st = 0; st < 2; ++st) {
-        rows_st[st] = job.n_rows - st * kTile;
-        rows_st[st] = rows_st[st] < 0 ? 0 : (rows_st[st] > kTile ? kTile : rows_st[st]);
-        pos0_st[st] = job.q_pos0 + st * kTile;
-        n_st[st] = 0;
-        if (rows_st[st] > 0) {
-            const int64_t last = pos0_st[st] + rows_st[st] - 1;
-            for (int t = 0; t < job.n_iv; ++t) {
-                int64_t end = job.iv_hi[t];
-                if (p.causal && end > last + 1) end = last + 1;
-                const int32_t c = end > job.iv_lo[t] ? (int32_t)((end - job.iv_lo[t] + kTile - 1) / kTile) : 0;
-                n_st[st] += c;
-                walk.cnt[t] = c > walk.cnt[t] ? c : walk.cnt[t];
+    // Thread 0 works out the CTA's geometry: heaviest (latest) causal tiles first; per stage the
+    // rows, positions and number of key tiles it takes part in.  Key tiles are walked interval 0
+    // first, then interval 1, in ascending position, so each stage's tiles are a prefix of the walk.
+    if (tid == 0) {
+        Geom g;
+        TileJob job;
+        g.found = locate_tile(p, (int64_t)gridDim.x - 1 - blockIdx.x, kBlockM, job) ? 1 : 0;
+        // An earlier CTA's wait expired: the launch is already lost, leave at once.
+        if (p.status && *reinterpret_cast<volatile int32_t *>(p.status) != 0) g.found = 0;
+        sh->abort_flag = 0;
+        if (g.found) {
+            g.q_row0 = (int32_t)job.q_row0; g.out_row0 = (int32_t)job.out_row0; g.kv_row0 = (int32_t)job.kv_row0;
+            g.cnt[0] = g.cnt[1] = 0;
+            for (int t = 0; t < 2; ++t) { g.lo[t] = (int32_t)job.iv_lo[t]; g.hi[t] = (int32_t)job.iv_hi[t]; }
+            for (int st = 0; st < 2; ++st) {
+                int32_t rows = job.n_rows - st * kTile;
+                rows = rows < 0 ? 0 : (rows > kTile ? kTile : rows);
+                g.rows[st] = rows;
+                g.pos0[st] = (int32_t)job.q_pos0 + st * kTile;
+                g.n[st] = 0;
+                if (rows > 0) {
+                    const int32_t last = g.pos0[st] + rows - 1;
+                    for (int t = 0; t < job.n_iv; ++t) {
+                        int32_t end = g.hi[t];
+                        if (p.causal && end > last + 1) end = last + 1;
+                        const int32_t c = end > g.lo[t] ? (end - g.lo[t] + kTile - 1) / kTile : 0;
+                        g.n[st] += c;
+                        g.cnt[t] = c > g.cnt[t] ? c : g.cnt[t];
+                    }
+                }
             }
+            g.n_max = g.cnt[0] + g.cnt[1];
         }
+        sh->g = g;
     }
-    const int n_max = walk.cnt[0] + walk.cnt[1];
+    __syncthreads();
+    if (!sh->g.found) return;
+    const int n_max = sh->g.n_max;
 
     if (tid == 0) {
         mbar_init(smem_u32(&sh->bar_q), 1);
@@ -155,16 +163,15 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             mbar_arrive_expect_tx(bar_q, 2 * kTileBytes);
 #pragma unroll
             for (int st = 0; st < 2; ++st) {
-                const int row = (int)(job.q_row0 + st * kTile);
+                const int row = sh->g.q_row0 + st * kTile;
                 tma_load_3d(sQ + st * kTileBytes, &tm_q, bar_q, 0, h, row);
                 tma_load_3d(sQ + st * kTileBytes + kHalfTileBytes, &tm_q, bar_q, 64, h, row);
             }
             for (int i = 0; i < 2 * n_max; ++i) {              // items: K(0), V(0), K(1), V(1), ...
                 const int slot = i % kStages, fill = i / kStages;
                 if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p.status)) break;
-                int64_t k0, hi_t;
-                walk.at(i >> 1, k0, hi_t);
-                const int krow = (int)(job.kv_row0 + k0);
+                const int jt = i >> 1, c0 = sh->g.cnt[0];
+                const int krow = sh->g.kv_row0 + (jt < c0 ? sh->g.lo[0] + jt * kTile : sh->g.lo[1] + (jt - c0) * kTile);
                 const uint32_t dst = sRing + slot * kTileBytes, bar = smem_u32(&sh->kv_full[slot]);
                 const void *map = (i & 1) ? (const void *)&tm_v : (const void *)&tm_k;
                 mbar_arrive_expect_tx(bar, kTileBytes);
@@ -204,6 +211,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                            smem_desc_sw128(b + ks * 2048u, kHalfTileBytes, 1024), idesc_pv, (accumulate || ks > 0) ? 1u : 0u);
             };
 
+            const int n_st[2] = {sh->g.n[0], sh->g.n[1]};
             bool ok = wait_bar(smem_u32(&sh->bar_q), 0, sh, p.status) && kv_wait(0);
             if (ok) {
                 if (n_st[0] > 0) issue_qk(0, 0);
@@ -231,39 +239,44 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
         }
         __syncwarp();
-    } else if (warp >= 8) {
+    } else if (warp >= kSoftmaxWarps) {
         reg_dealloc<kLightRegs>();
     } else {
         // ------------------------------------------------------------------ softmax + epilogue
         reg_alloc<kSoftmaxRegs>();
-        const int st = warp >> 2;
-        const int row_in_tile = (warp & 3) * 32 + lane;
-        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const int st = warp >> 2, quarter = warp & 3;
+        const int row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
         const uint32_t tS = tmem + lane_base + kColS + st * kTile;
         const uint32_t tO = tmem + lane_base + kColO + st * kTile;
-        const int64_t my_pos = pos0_st[st] + row_in_tile;
-        const int n_mine = n_st[st];
+        const int n_mine = sh->g.n[st];
         const uint32_t bar_s = smem_u32(&sh->s_full[st]), bar_p = smem_u32(&sh->p_ready[st]);
+        // Per interval: where it ends, and the first key position that some row of this stage cannot
+        // see (tiles reaching past it need the mask).
+        const int pos0 = sh->g.pos0[st], my_pos = pos0 + row_in_tile, cnt0 = sh->g.cnt[0];
+        int iv_full[2], iv_mine[2];
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const int hi_t = sh->g.hi[t];
+            iv_full[t] = (p.causal && pos0 + 1 < hi_t) ? pos0 + 1 : hi_t;
+            iv_mine[t] = (p.causal && my_pos + 1 < hi_t) ? my_pos + 1 : hi_t;
+        }
+        int k0 = sh->g.lo[0], cur = 0;
 
         float m_ref = -INFINITY, l_run = 0.f;                // m_ref in log2 units of the scaled scores
         bool ok = true;
-        for (int j = 0; j < n_mine; ++j) {
+        for (int j = 0; j < n_mine; ++j, k0 += kTile) {
+            if (j == cnt0) { cur = 1; k0 = sh->g.lo[1]; }
             ok = __all_sync(0xffffffffu, wait_bar(bar_s, j & 1, sh, p.status));     // warp-uniform
             if (!ok) break;
             tc_fence_after();
 
             uint32_t r[kTile];
             tmem_ld128(tS, r);
-            int64_t k0, hi_t;
-            walk.at(j, k0, hi_t);
             // Mask only when some row of this stage cannot see the whole tile.
-            int64_t full_lim = hi_t;
-            if (p.causal && pos0_st[st] + 1 < full_lim) full_lim = pos0_st[st] + 1;
-            const bool masked = k0 + kTile > full_lim;
+            const bool masked = k0 + kTile > (cur ? iv_full[1] : iv_full[0]);
             if (masked) {
-                int64_t lim = hi_t;
-                if (p.causal && my_pos + 1 < lim) lim = my_pos + 1;
-                int n_vis = (int)(lim - k0);
+                int n_vis = (cur ? iv_mine[1] : iv_mine[0]) - k0;
                 n_vis = n_vis < 0 ? 0 : (n_vis > kTile ? kTile : n_vis);
 #pragma unroll
                 for (int c = 0; c < kTile; ++c) r[c] = (c < n_vis) ? r[c] : 0xff800000u;   // -inf
@@ -323,12 +336,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
             const float2 s01 = __fadd2_rn(__fadd2_rn(sum[0], sum[1]), __fadd2_rn(sum[2], sum[3]));
             l_run += s01.x + s01.y;
-            {
-                uint32_t(&lo)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[0]);
-                uint32_t(&hi)[32] = *reinterpret_cast<uint32_t(*)[32]>(&r[32]);
-                tmem_st32(tS, lo);
-                tmem_st32(tS + 32, hi);
-            }
+            tmem_st32(tS, r);
+            tmem_st32(tS + 32, r + 32);
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
@@ -337,12 +346,12 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
         // Epilogue: O / l and LSE = ln2 * m + ln l; rows without any visible key give 0 and -inf.
         if (ok && n_mine > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->o_final[st]), 0, sh, p.status));
-        if (ok && rows_st[st] > 0) {
+        if (ok && sh->g.rows[st] > 0) {
             tc_fence_after();
-            const bool valid = row_in_tile < rows_st[st];
+            const bool valid = row_in_tile < sh->g.rows[st];
             const bool empty = (l_run == 0.f);
             const float inv = empty ? 0.f : 1.f / l_run;
-            const int64_t row = job.out_row0 + st * kTile + row_in_tile;
+            const int64_t row = (int64_t)sh->g.out_row0 + st * kTile + row_in_tile;
             const int64_t obase = (row * p.Hq + h) * kHeadDim;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -425,6 +434,10 @@ int launch_attn_bf16(const AttnParams &p, cudaStream_t stream)
         kv_rows = 0;
         for (int t = 0; t < p.n_iv; ++t) kv_rows = p.iv_hi[t] > kv_rows ? p.iv_hi[t] : kv_rows;
     }
+    if (q_rows >= ((int64_t)1 << 31) || kv_rows >= ((int64_t)1 << 31)) {
+        set_error("pec_prefill_attn: more than 2^31 rows unsupported");
+        return PEC_ERR_UNSUPPORTED;
+    }
     CUtensorMap tm_q, tm_k, tm_v;
     if (!make_map(&tm_q, p.q, q_rows, p.Hq, p.q_stride_t, p.q_stride_h) ||
         !make_map(&tm_k, p.k, kv_rows, p.Hkv, p.k_stride_t, p.k_stride_h) ||
@@ -434,6 +447,14 @@ int launch_attn_bf16(const AttnParams &p, cudaStream_t stream)
     }
     if (cudaFuncSetAttribute(attn_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) {
         set_error("pec_prefill_attn: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
+        return PEC_ERR_CUDA;
+    }
+    // The softmax warpgroups take registers the third warpgroup gives up; that only works when the
+    // launch allocation (registers per thread x threads) covers the new split.
+    cudaFuncAttributes attr;
+    if (cudaFuncGetAttributes(&attr, attn_bf16_kernel) != cudaSuccess ||
+        attr.numRegs * kThreads < kSoftmaxWarps * 32 * kSoftmaxRegs + (kThreads - kSoftmaxWarps * 32) * kLightRegs) {
+        set_error("pec_prefill_attn: kernel register allocation too small for the warp-role register split");
         return PEC_ERR_CUDA;
     }
     int64_t tiles = (p.total_rows + kBlockM - 1) / kBlockM;
