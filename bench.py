@@ -115,7 +115,7 @@ def run_reference(args, wl):
     if rank != 0:
         return
     q, k, v = workloads.qkv(wl.seed, wl.seq_len, wl.hq, wl.hkv, 128, wl.dtype)
-    per_step = max(2.0, min(20.0, 90.0 / (args.steps + args.warmup)))
+    per_step = args.reference_seconds or max(2.0, min(20.0, 90.0 / (args.steps + args.warmup)))
     for _ in range(args.warmup):
         oracle_sample(wl, q, k, v, target_s=per_step)
     res = [oracle_sample(wl, q, k, v, target_s=per_step) for _ in range(args.steps)]
@@ -141,6 +141,25 @@ def workload_config(wl):
             "flops": "4*D*Hq*(exact causal pairs), attention only, single layer"}
 
 
+# ----------------------------------------------------------------------------- multi-rank plumbing
+def replica_seed(wl, rank):
+    """Replicas only: rank r runs the same single-GPU workload on its own seeded request."""
+    return wl.seed + 1000 * rank
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of per-rank timings (every rank gets the result)."""
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_tflops(flops_per_replica_step, world, ms_per_step):
+    """All replicas' work over the slowest rank's time."""
+    return world * flops_per_replica_step / (ms_per_step * 1e-3) / 1e12
+
+
 # ----------------------------------------------------------------------------- GPU arm
 def run_ours(args, wl):
     from paper_2409_15104_b200 import binding
@@ -158,7 +177,7 @@ def run_ours(args, wl):
     binding.load()
 
     # Replicas only: every rank runs the same single-GPU workload on its own seeded request.
-    seed = wl.seed + 1000 * rank
+    seed = replica_seed(wl, rank)
     q_h, k_h, v_h = workloads.qkv(seed, wl.seq_len, wl.hq, wl.hkv, 128, wl.dtype)
     q_h, k_h, v_h = q_h.pin_memory(), k_h.pin_memory(), v_h.pin_memory()
     q, k, v = q_h.to(dev), k_h.to(dev), v_h.to(dev)
@@ -226,10 +245,7 @@ def run_ours(args, wl):
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
     binding.check_status()
 
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(times[0]), float(times[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, dev)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -239,7 +255,7 @@ def run_ours(args, wl):
     pairs = workloads.causal_pairs(wl.seq_len)
     flops_step = workloads.attention_flops(pairs, wl.hq)
     ms_step = total_ms / args.steps
-    tflops = world * flops_step / (ms_step * 1e-3) / 1e12
+    tflops = whole_job_tflops(flops_step, world, ms_step)
     attn_avg_ms = sum(attn_ms) / len(attn_ms)
     flops_launch = flops_step / wl.num_parts          # zigzag partitions carry equal pair counts
     attn_tflops = flops_launch / (attn_avg_ms * 1e-3) / 1e12
@@ -274,7 +290,7 @@ def run_ours(args, wl):
                          "sample": f"{cpu['rows']} seeded random query rows x {wl.hq} heads of the same request, "
                                    f"{cpu['seconds']:.1f} s; tokens/s extrapolated by pair count: "
                                    f"{cpu['tokens_per_s_extrapolated']:.3f}"},
-        "e2e": {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+        "e2e": {"value": whole_job_tflops(flops_step, world, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": args.steps * runner.launches_per_step(),
         "clocks": clocks,
@@ -291,6 +307,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=["c3", "c5"], default="c3")
+    ap.add_argument("--reference-seconds", type=float, default=0.0,
+                    help="--impl reference: CPU seconds per step (default: 90 s spread over the steps, 2-20 s each)")
     ap.add_argument("--profile", action="store_true",
                     help="profiling runs: skip the end-to-end and CPU-baseline legs (the printed line is not a result)")
     args = ap.parse_args()
