@@ -218,7 +218,8 @@ def run_ours(args, wl):
             print(json.dumps({"profile_run": True, "ms_per_step": total_ms / args.steps,
                               "attn_ms_per_launch": sum(attn_ms) / len(attn_ms),
                               "attn_tflops": fl / wl.num_parts / (sum(attn_ms) / len(attn_ms)) / 1e9,
-                              "merge_ms_per_launch": (sum(merge_ms) / len(merge_ms)) if merge_ms else None}), flush=True)
+                              "merge_ms_per_launch": (sum(merge_ms) / len(merge_ms)) if merge_ms else None,
+                              "clocks": clocks}), flush=True)
         if dist is not None:
             dist.destroy_process_group()
         return
