@@ -2,7 +2,8 @@
 """Benchmark of the partial causal prefill attention path on B200.
 
 A step is one pass of the whole path over one synthetic long request: host plan, one partial
-attention launch per zigzag KV partition, running LSE merges, final output in the input dtype.
+attention launch per zigzag KV partition, LSE merge of the partials (n-way per group of resident
+partials), final output in the input dtype.
 Prints one JSON line (see --help for the knobs).  `--impl reference` times the fp64 CPU oracle
 on a bounded sample of the same workload instead.
 """
@@ -263,11 +264,18 @@ def run_ours(args, wl):
     items = wl.seq_len * wl.hq
     merge = None
     if merge_ms:
-        merge_avg = sum(merge_ms) / len(merge_ms)
-        merge = {"ms_per_launch": merge_avg, "algorithmic_gbs": items * 1548 / (merge_avg * 1e-3) / 1e9,
-                 "bytes_per_item": 1548, "frac_of_measured_hbm": items * 1548 / (merge_avg * 1e-3) / 1e9 / peaks["hbm"],
-                 "frac_of_nominal_8TBs": items * 1548 / (merge_avg * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-                 "note": "upper bound on bytes: rows whose side-b partial is empty are skipped by the in-place merge"}
+        # Algorithmic bytes of one merge launch over n parts: n reads of (128*4 + 4) B per (row, head) plus one
+        # write (fp32 partial: 516 B; final bf16 output + LSE: 260 B).  Rows of a part with no visible key are
+        # skipped by the kernels, so this is an upper bound on the traffic.
+        per_step = len(runner.merge_parts)
+        out_final = 128 * (2 if wl.dtype == torch.bfloat16 else 4) + 4
+        byts = [items * (n * 516 + (out_final if i == per_step - 1 else 516)) for i, n in enumerate(runner.merge_parts)]
+        total_bytes = sum(byts) * args.steps
+        gbs = total_bytes / (sum(merge_ms) * 1e-3) / 1e9
+        merge = {"launches_per_step": per_step, "parts_per_launch": runner.merge_parts,
+                 "ms_per_launch": sum(merge_ms) / len(merge_ms), "algorithmic_gbs": gbs,
+                 "frac_of_measured_hbm": gbs / peaks["hbm"], "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+                 "note": "bytes are an upper bound: rows of a part with no visible key are not read"}
     h2d = q_h.numel() * q_h.element_size() + 2 * k_h.numel() * k_h.element_size()
     d2h = o_h.numel() * o_h.element_size() + l_h.numel() * 4
 

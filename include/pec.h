@@ -134,6 +134,22 @@ int pec_attn_merge(const void *o_a, const float *lse_a, const void *o_b, const f
                    int32_t part_dtype, int32_t out_dtype, void *cuda_stream);
 
 /*
+ * The same merge over n partials at once (2 <= n <= PEC_MERGE_MAX_PARTS): one pass over
+ * memory instead of n-1, which is what a rank holding several ring steps' partials, or a
+ * single GPU running virtual partitions, wants (Section 2.2):
+ *     lse = ln sum_i exp(lse_i);   o = sum_i exp(lse_i - lse) * o_i
+ * o_parts / lse_parts: HOST arrays of n DEVICE pointers ([rows, Hq, D] fp32 and [rows, Hq]
+ * fp32, contiguous, 16-byte aligned); the arrays are read during the call only.  o_out /
+ * lse_out as in pec_attn_merge; they may alias part 0 (both, fp32 output) and no other part.
+ * Parts whose lse is -inf for a row are not read for that row.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.
+ */
+#define PEC_MERGE_MAX_PARTS 16
+int pec_attn_merge_n(const void *const *o_parts, const float *const *lse_parts, int32_t n,
+                     void *o_out, float *lse_out, int64_t rows, int32_t Hq, int32_t D,
+                     int32_t part_dtype, int32_t out_dtype, void *cuda_stream);
+
+/*
  * Host-side plan of how a request of seq_len tokens is split.  All arrays are
  * host memory owned by the caller; an array pointer may be NULL to skip that
  * output.  Capacities are element counts; the needed counts are always written

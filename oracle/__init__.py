@@ -8,6 +8,7 @@ from .reference import (  # noqa: F401
     prefill_attn,
     varlen_attn,
     merge,
+    merge_n,
     plan_partitions,
     partition_intervals,
     oracle_threads,

@@ -220,3 +220,22 @@ def merge(o_a, lse_a, o_b, lse_b):
     cb = np.where(both_empty, 0.0, wb / np.where(both_empty, 1.0, tot))
     o = ca[..., None] * o_a + cb[..., None] * o_b
     return o, lse
+
+
+def merge_n(o_parts, lse_parts):
+    """Combine n partial results over pairwise disjoint key sets in one step (fp64 numpy):
+    LSE = ln sum_i exp(LSE_i); O = sum_i exp(LSE_i - LSE) O_i.  Rows where every part is empty
+    give (0, -inf)."""
+    o_parts = [np.asarray(o, dtype=np.float64) for o in o_parts]
+    ls = np.stack([np.asarray(l, dtype=np.float64) for l in lse_parts])       # [n, rows, H]
+    m = ls.max(axis=0)
+    empty = np.isneginf(m)
+    m_safe = np.where(empty, 0.0, m)
+    w = np.exp(ls - m_safe)                                                    # exp(-inf) = 0
+    tot = w.sum(axis=0)
+    lse = np.where(empty, -np.inf, m_safe + np.log(np.where(empty, 1.0, tot)))
+    o = np.zeros_like(o_parts[0])
+    for i, oi in enumerate(o_parts):
+        c = np.where(empty, 0.0, w[i] / np.where(empty, 1.0, tot))
+        o += c[..., None] * np.where(c[..., None] == 0.0, 0.0, oi)
+    return o, lse

@@ -62,7 +62,9 @@ class pec_plan(ctypes.Structure):
     ]
 
 
-EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_plan_partitions", "pec_last_error")
+EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_attn_merge_n", "pec_plan_partitions",
+           "pec_last_error")
+PEC_MERGE_MAX_PARTS = 16
 
 
 def load():
@@ -81,6 +83,10 @@ def load():
     lib.pec_attn_merge.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                    ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32,
                                    ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
+    lib.pec_attn_merge_n.restype = ctypes.c_int
+    lib.pec_attn_merge_n.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p), ctypes.c_int32,
+                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32,
+                                     ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
     lib.pec_plan_partitions.restype = ctypes.c_int
     lib.pec_plan_partitions.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, ctypes.c_int32,
                                         ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(pec_plan)]
@@ -205,6 +211,28 @@ def pec_attn_merge(o_a, lse_a, o_b, lse_b, *, out_dtype=torch.float32, o_out=Non
     _check(lib.pec_attn_merge(o_a.data_ptr(), lse_a.data_ptr(), o_b.data_ptr(), lse_b.data_ptr(),
                               o_out.data_ptr(), lse_out.data_ptr(), rows, Hq, D,
                               _dtype_code(o_a.dtype), _dtype_code(o_out.dtype), _stream_ptr(stream)))
+    return o_out, lse_out
+
+
+def pec_attn_merge_n(o_parts, lse_parts, *, out_dtype=torch.float32, o_out=None, lse_out=None, inplace=False,
+                     stream=None):
+    """Merge n fp32 partials of the same rows in one pass; returns (o, lse).  inplace=True writes into part 0."""
+    lib = load()
+    n = len(o_parts)
+    assert n == len(lse_parts)
+    rows, Hq, D = o_parts[0].shape
+    for t in list(o_parts) + list(lse_parts):
+        assert t.is_cuda and t.is_contiguous()
+    if inplace:
+        o_out, lse_out = o_parts[0], lse_parts[0]
+    if o_out is None:
+        o_out = torch.empty((rows, Hq, D), dtype=out_dtype, device=o_parts[0].device)
+    if lse_out is None:
+        lse_out = torch.empty((rows, Hq), dtype=torch.float32, device=o_parts[0].device)
+    op = (ctypes.c_void_p * n)(*[t.data_ptr() for t in o_parts])
+    lp = (ctypes.c_void_p * n)(*[t.data_ptr() for t in lse_parts])
+    _check(lib.pec_attn_merge_n(op, lp, n, o_out.data_ptr(), lse_out.data_ptr(), rows, Hq, D,
+                                _dtype_code(o_parts[0].dtype), _dtype_code(o_out.dtype), _stream_ptr(stream)))
     return o_out, lse_out
 
 

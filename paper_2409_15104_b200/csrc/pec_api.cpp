@@ -151,3 +151,32 @@ extern "C" int pec_attn_merge(const void *o_a, const float *lse_a, const void *o
                         o_out, lse_out, rows * (int64_t)Hq, out_dtype == PEC_BF16, alias_o ? 1 : 0,
                         static_cast<cudaStream_t>(cuda_stream));
 }
+
+extern "C" int pec_attn_merge_n(const void *const *o_parts, const float *const *lse_parts, int32_t n,
+                                void *o_out, float *lse_out, int64_t rows, int32_t Hq, int32_t D,
+                                int32_t part_dtype, int32_t out_dtype, void *cuda_stream)
+{
+    if (!o_parts || !lse_parts || !o_out || !lse_out) { set_error("pec_attn_merge_n: NULL pointer"); return PEC_ERR_INVALID_ARG; }
+    if (n < 2 || n > PEC_MERGE_MAX_PARTS) { set_error("pec_attn_merge_n: need 2 <= n <= %d (got %d)", PEC_MERGE_MAX_PARTS, n); return PEC_ERR_INVALID_ARG; }
+    if (rows < 0 || Hq < 1) { set_error("pec_attn_merge_n: need rows >= 0 and Hq >= 1"); return PEC_ERR_INVALID_ARG; }
+    if (D != kHeadDim) { set_error("pec_attn_merge_n: D=%d unsupported (only 128)", D); return PEC_ERR_UNSUPPORTED; }
+    if (part_dtype != PEC_F32) { set_error("pec_attn_merge_n: partials must be fp32"); return PEC_ERR_UNSUPPORTED; }
+    if (out_dtype != PEC_F32 && out_dtype != PEC_BF16) { set_error("pec_attn_merge_n: unknown out_dtype %d", out_dtype); return PEC_ERR_UNSUPPORTED; }
+    MergeParts parts;
+    parts.n = n;
+    for (int k = 0; k < PEC_MERGE_MAX_PARTS; ++k) { parts.o[k] = nullptr; parts.lse[k] = nullptr; }
+    for (int k = 0; k < n; ++k) {
+        if (!o_parts[k] || !lse_parts[k]) { set_error("pec_attn_merge_n: part %d is NULL", k); return PEC_ERR_INVALID_ARG; }
+        if (!aligned16(o_parts[k]) || !aligned16(lse_parts[k])) { set_error("pec_attn_merge_n: buffers must be 16-byte aligned"); return PEC_ERR_ALIGNMENT; }
+        parts.o[k] = static_cast<const float *>(o_parts[k]);
+        parts.lse[k] = lse_parts[k];
+        const bool alias_o = (o_out == o_parts[k]), alias_l = (lse_out == lse_parts[k]);
+        if ((alias_o || alias_l) && (k != 0 || alias_o != alias_l || out_dtype != PEC_F32)) {
+            set_error("pec_attn_merge_n: outputs may alias part 0 only (both o and lse, fp32 output)");
+            return PEC_ERR_INVALID_ARG;
+        }
+    }
+    if (!aligned16(o_out) || !aligned16(lse_out)) { set_error("pec_attn_merge_n: buffers must be 16-byte aligned"); return PEC_ERR_ALIGNMENT; }
+    if (rows == 0) return PEC_OK;
+    return launch_merge_n(parts, o_out, lse_out, rows * (int64_t)Hq, out_dtype == PEC_BF16, static_cast<cudaStream_t>(cuda_stream));
+}

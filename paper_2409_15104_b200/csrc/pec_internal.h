@@ -44,4 +44,12 @@ int launch_merge(const float *o_a, const float *lse_a, const float *o_b, const f
                  void *o_out, float *lse_out, int64_t items, int out_is_bf16, int inplace,
                  cudaStream_t stream);
 
+struct MergeParts {
+    const float *o[PEC_MERGE_MAX_PARTS];
+    const float *lse[PEC_MERGE_MAX_PARTS];
+    int32_t n;
+};
+int launch_merge_n(const MergeParts &parts, void *o_out, float *lse_out, int64_t items, int out_is_bf16,
+                   cudaStream_t stream);
+
 }  // namespace pec

@@ -91,9 +91,86 @@ merge_kernel(const float *o_a, const float *lse_a, const float *__restrict__ o_b
     }
 }
 
-int launch_merge(const float *o_a, const float *lse_a, const float *o_b, const float *lse_b,
-                 void *o_out, float *lse_out, int64_t items, int out_is_bf16, int inplace,
-                 cudaStream_t stream)
+// n-way form: lane i takes the n LSE values of item i, turns them into n weights (registers), and
+// the weights of each item are again broadcast by shuffles while the lanes stream that item's
+// channels from every part with a non-zero weight.  Bytes per item: at most (n + 1) * 516.
+// The output may alias part 0: each item is read before it is written, by the same warp.
+template <bool kOutBf16>
+__global__ void __launch_bounds__(kMergeThreads)
+merge_n_kernel(const MergeParts parts, void *o_out, float *lse_out, int64_t items)
+{
+    const int lane = threadIdx.x & 31;
+    const int n = parts.n;
+    const int64_t warp = ((int64_t)blockIdx.x * kMergeThreads + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * kMergeThreads) >> 5;
+    const int64_t n_groups = (items + kItemsPerWarp - 1) / kItemsPerWarp;
+
+    for (int64_t g = warp; g < n_groups; g += n_warps) {
+        const int64_t base = g * kItemsPerWarp;
+        const int64_t mine = base + lane;
+        float w[PEC_MERGE_MAX_PARTS];
+#pragma unroll
+        for (int k = 0; k < PEC_MERGE_MAX_PARTS; ++k) w[k] = 0.f;
+        if (mine < items) {
+            float m = -INFINITY;
+#pragma unroll
+            for (int k = 0; k < PEC_MERGE_MAX_PARTS; ++k)
+                if (k < n) { w[k] = parts.lse[k][mine]; m = fmaxf(m, w[k]); }
+            float lse = -INFINITY;
+            if (m != -INFINITY) {
+                float tot = 0.f;
+#pragma unroll
+                for (int k = 0; k < PEC_MERGE_MAX_PARTS; ++k)
+                    if (k < n) { w[k] = expf(w[k] - m); tot += w[k]; }     // the largest one is exactly 1
+                const float inv = 1.f / tot;
+#pragma unroll
+                for (int k = 0; k < PEC_MERGE_MAX_PARTS; ++k) w[k] *= inv;
+                lse = m + logf(tot);
+            } else {
+#pragma unroll
+                for (int k = 0; k < PEC_MERGE_MAX_PARTS; ++k) w[k] = 0.f;
+            }
+            lse_out[mine] = lse;
+        }
+        const int n_here = (items - base) < kItemsPerWarp ? (int)(items - base) : kItemsPerWarp;
+#pragma unroll 2
+        for (int i = 0; i < n_here; ++i) {
+            const int64_t off = (base + i) * (kHeadDim / 4) + lane;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            // four parts at a time: all their loads are issued before the first is used
+#pragma unroll
+            for (int k0 = 0; k0 < PEC_MERGE_MAX_PARTS; k0 += 4) {
+                if (k0 < n) {                                  // warp-uniform
+                    float f[4];
+                    float4 v[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        f[u] = (k0 + u < n) ? __shfl_sync(0xffffffffu, w[k0 + u], i) : 0.f;
+                        v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (f[u] != 0.f) v[u] = ld_stream(reinterpret_cast<const float4 *>(parts.o[k0 + u]) + off);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        acc.x = fmaf(f[u], v[u].x, acc.x); acc.y = fmaf(f[u], v[u].y, acc.y);
+                        acc.z = fmaf(f[u], v[u].z, acc.z); acc.w = fmaf(f[u], v[u].w, acc.w);
+                    }
+                }
+            }
+            if (kOutBf16) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y);
+                __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z, acc.w);
+                uint2 pk;
+                pk.x = *reinterpret_cast<uint32_t *>(&lo);
+                pk.y = *reinterpret_cast<uint32_t *>(&hi);
+                reinterpret_cast<uint2 *>(o_out)[off] = pk;
+            } else {
+                reinterpret_cast<float4 *>(o_out)[off] = acc;
+            }
+        }
+    }
+}
+
+static int merge_grid(int64_t items, const char *who, int64_t *ctas_out)
 {
     static int sm_count = 0;
     if (sm_count == 0) {
@@ -101,15 +178,38 @@ int launch_merge(const float *o_a, const float *lse_a, const float *o_b, const f
         if (cudaGetDevice(&dev) != cudaSuccess ||
             cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0) {
             sm_count = 0;
-            set_error("pec_attn_merge: cannot query the device: %s", cudaGetErrorString(cudaGetLastError()));
+            set_error("%s: cannot query the device: %s", who, cudaGetErrorString(cudaGetLastError()));
             return PEC_ERR_CUDA;
         }
     }
     const int64_t n_groups = (items + kItemsPerWarp - 1) / kItemsPerWarp;
     const int64_t warps_per_cta = kMergeThreads / 32;
     int64_t ctas = (n_groups + warps_per_cta - 1) / warps_per_cta;
-    const int64_t cap = (int64_t)sm_count * 8;          // 8 resident CTAs of 256 threads per SM
-    if (ctas > cap) ctas = cap;
+    const int64_t cap = (int64_t)sm_count * 8;
+    *ctas_out = ctas > cap ? cap : ctas;
+    return PEC_OK;
+}
+
+int launch_merge_n(const MergeParts &parts, void *o_out, float *lse_out, int64_t items, int out_is_bf16,
+                   cudaStream_t stream)
+{
+    int64_t ctas = 0;
+    const int rc = merge_grid(items, "pec_attn_merge_n", &ctas);
+    if (rc != PEC_OK) return rc;
+    if (out_is_bf16) merge_n_kernel<true><<<(unsigned)ctas, kMergeThreads, 0, stream>>>(parts, o_out, lse_out, items);
+    else             merge_n_kernel<false><<<(unsigned)ctas, kMergeThreads, 0, stream>>>(parts, o_out, lse_out, items);
+    const cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) { set_error("pec_attn_merge_n: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
+    return PEC_OK;
+}
+
+int launch_merge(const float *o_a, const float *lse_a, const float *o_b, const float *lse_b,
+                 void *o_out, float *lse_out, int64_t items, int out_is_bf16, int inplace,
+                 cudaStream_t stream)
+{
+    int64_t ctas = 0;
+    const int rc = merge_grid(items, "pec_attn_merge", &ctas);
+    if (rc != PEC_OK) return rc;
     if (out_is_bf16)  merge_kernel<true, false><<<(unsigned)ctas, kMergeThreads, 0, stream>>>(o_a, lse_a, o_b, lse_b, o_out, lse_out, items);
     else if (inplace) merge_kernel<false, true><<<(unsigned)ctas, kMergeThreads, 0, stream>>>(o_a, lse_a, o_b, lse_b, o_out, lse_out, items);
     else              merge_kernel<false, false><<<(unsigned)ctas, kMergeThreads, 0, stream>>>(o_a, lse_a, o_b, lse_b, o_out, lse_out, items);

@@ -14,46 +14,75 @@ from . import binding
 
 
 class PartitionedPrefill:
-    """Buffers and call sequence for P virtual sequence partitions merged through their LSE."""
+    """Buffers and call sequence for P virtual sequence partitions merged through their LSE.
 
-    def __init__(self, seq_len, hq, num_parts, dtype, device, part_align=128):
+    Partials are kept in up to `max_live` fp32 buffers (bounded by `partial_budget_bytes`) and
+    merged with one n-way pass per group instead of P-1 two-way passes; with two buffers this
+    degenerates to the running two-way merge.
+    """
+
+    def __init__(self, seq_len, hq, num_parts, dtype, device, part_align=128, partial_budget_bytes=24 << 30):
         self.S, self.Hq, self.P, self.align = seq_len, hq, num_parts, part_align
         self.dtype = dtype
         f32 = torch.float32
-        self.acc_o = torch.empty((seq_len, hq, 128), dtype=f32, device=device)
-        self.acc_l = torch.empty((seq_len, hq), dtype=f32, device=device)
-        if num_parts > 1:
-            self.tmp_o = torch.empty_like(self.acc_o)
-            self.tmp_l = torch.empty_like(self.acc_l)
+        per_partial = seq_len * hq * (128 * 4 + 4)
+        self.max_live = max(2, min(num_parts, binding.PEC_MERGE_MAX_PARTS, partial_budget_bytes // max(per_partial, 1)))
+        n_buf = self.max_live if num_parts > 1 else 0
+        self.part_o = [torch.empty((seq_len, hq, 128), dtype=f32, device=device) for _ in range(n_buf)]
+        self.part_l = [torch.empty((seq_len, hq), dtype=f32, device=device) for _ in range(n_buf)]
         self.out_o = torch.empty((seq_len, hq, 128), dtype=dtype, device=device)
         self.out_l = torch.empty((seq_len, hq), dtype=f32, device=device)
         self.attn_events = []      # (start, end) CUDA events per attention launch when timing
         self.merge_events = []
+        self.merge_parts = []      # parts merged by each merge launch of the last run
+
+    def merge_launches(self):
+        """Merge launches per step: the first group holds max_live partials, later ones max_live-1 new ones."""
+        if self.P == 1:
+            return 0
+        rest = self.P - self.max_live
+        return 1 + (0 if rest <= 0 else -(-rest // (self.max_live - 1)))
 
     def launches_per_step(self):
-        return self.P + (self.P - 1) if self.P > 1 else 1
+        return self.P + self.merge_launches()
 
     def run(self, q, k, v, stream=None, time_kernels=False):
         """Returns (o [S,Hq,128] in the input dtype, lse [S,Hq] fp32)."""
         P = self.P
-        plan = binding.pec_plan_partitions(self.S, P, 0, self.align, 128, 128, True, tiles=False)
-        self.plan = plan
+        self.plan = binding.pec_plan_partitions(self.S, P, 0, self.align, 128, 128, True, tiles=False)
+        self.merge_parts = []
         if P == 1:
             self._attn(q, k, v, 0, self.out_o, self.out_l, stream, time_kernels)
             return self.out_o, self.out_l
-        for p in range(P):
-            o, l = (self.acc_o, self.acc_l) if p == 0 else (self.tmp_o, self.tmp_l)
-            self._attn(q, k, v, p, o, l, stream, time_kernels)
-            if p == 0:
-                continue
+        p = 0
+        first = True
+        while p < P:
+            # buffer 0 holds the running result after the first group
+            slots = list(range(0 if first else 1, self.max_live))
+            used = []
+            for b in slots:
+                if p >= P:
+                    break
+                self._attn(q, k, v, p, self.part_o[b], self.part_l[b], stream, time_kernels)
+                used.append(b)
+                p += 1
+            group = used if first else [0] + used
+            last = p >= P
             ev = self._events(time_kernels, self.merge_events, stream)
-            if p < P - 1:
-                binding.pec_attn_merge(self.acc_o, self.acc_l, o, l, inplace=True, stream=stream)
+            o_parts, l_parts = [self.part_o[b] for b in group], [self.part_l[b] for b in group]
+            if len(group) == 2 and not last:
+                binding.pec_attn_merge(o_parts[0], l_parts[0], o_parts[1], l_parts[1], inplace=True, stream=stream)
+            elif len(group) == 2:
+                binding.pec_attn_merge(o_parts[0], l_parts[0], o_parts[1], l_parts[1], o_out=self.out_o,
+                                       lse_out=self.out_l, stream=stream)
+            elif last:
+                binding.pec_attn_merge_n(o_parts, l_parts, o_out=self.out_o, lse_out=self.out_l, stream=stream)
             else:
-                binding.pec_attn_merge(self.acc_o, self.acc_l, o, l, o_out=self.out_o, lse_out=self.out_l,
-                                       stream=stream)
+                binding.pec_attn_merge_n(o_parts, l_parts, inplace=True, stream=stream)
             if ev:
                 ev[1].record(stream)
+            self.merge_parts.append(len(group))
+            first = False
         return self.out_o, self.out_l
 
     def _events(self, on, store, stream):

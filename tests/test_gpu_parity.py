@@ -50,6 +50,26 @@ def test_merge_ignores_garbage_behind_an_empty_side(pec):
     assert torch.equal(o.cpu(), oa) and torch.equal(l.cpu(), la)
 
 
+@pytest.mark.parametrize("n", [2, 3, 8, 16])
+@pytest.mark.parametrize("mode", ["f32", "bf16", "inplace"])
+def test_merge_n_matches_oracle(pec, n, mode):
+    rows, hq = 517, 3
+    g = torch.Generator().manual_seed(n * 17 + len(mode))
+    os_ = [torch.randn(rows, hq, 128, generator=g) for _ in range(n)]
+    ls_ = [torch.randn(rows, hq, generator=g) * 4 for _ in range(n)]
+    for i in range(n):                                  # empty rows, different per part; rows 0..4 empty everywhere
+        ls_[i][i::n + 1] = float("-inf"); os_[i][i::n + 1] = float("nan")
+        ls_[i][:5] = float("-inf")
+    want = oracle.merge_n([o.numpy() for o in os_], [l.numpy() for l in ls_])
+    do, dl = [o.to(DEV) for o in os_], [l.to(DEV) for l in ls_]
+    if mode == "inplace":
+        o, l = pec.pec_attn_merge_n(do, dl, inplace=True)
+        assert o.data_ptr() == do[0].data_ptr()
+    else:
+        o, l = pec.pec_attn_merge_n(do, dl, out_dtype=torch.float32 if mode == "f32" else torch.bfloat16)
+    compare(o, l, *want, 2e-2 if mode == "bf16" else 1e-5, 1e-5, f"merge_n n={n} {mode}")
+
+
 # ------------------------------------------------------------------ attention, single request
 SHAPES = [  # (S, Hq, Hkv)
     (1, 1, 1), (2, 2, 1), (63, 2, 2), (64, 4, 2), (65, 2, 1), (127, 4, 4), (128, 8, 2), (129, 2, 2),

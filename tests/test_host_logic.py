@@ -109,3 +109,24 @@ def test_merge_validates_on_the_host():
     assert f(ok[0], ok[1], ok[2], ok[3], ok[0], ok[5], 4, 2, 128, 2, 2, None) == -1   # o aliased, lse not
     assert f(ok[0], ok[1], ok[2], ok[3], ok[2], ok[3], 4, 2, 128, 2, 2, None) == -1   # aliasing side b
     assert f(*ok, 0, 2, 128, 2, 2, None) == 0                                          # nothing to do
+
+
+def test_merge_n_validates_on_the_host():
+    lib = binding.load()
+    f = lib.pec_attn_merge_n
+
+    def ptrs(vals):
+        return (ctypes.c_void_p * len(vals))(*vals)
+
+    o3, l3 = ptrs([4096, 8192, 12288]), ptrs([16384, 20480, 24576])
+    assert f(o3, l3, 3, 32768, 36864, 0, 2, 128, 2, 2, None) == 0            # nothing to do
+    assert f(o3, l3, 1, 32768, 36864, 4, 2, 128, 2, 2, None) == -1           # n too small
+    assert f(o3, l3, 17, 32768, 36864, 4, 2, 128, 2, 2, None) == -1          # n too large
+    assert f(None, l3, 3, 32768, 36864, 4, 2, 128, 2, 2, None) == -1
+    assert f(o3, l3, 3, 32768, 36864, 4, 2, 64, 2, 2, None) == -2
+    assert f(o3, l3, 3, 32768, 36864, 4, 2, 128, 1, 2, None) == -2
+    assert f(ptrs([4100, 8192, 12288]), l3, 3, 32768, 36864, 4, 2, 128, 2, 2, None) == -3
+    assert f(o3, l3, 3, 8192, 20480, 4, 2, 128, 2, 2, None) == -1            # aliasing part 1
+    assert f(o3, l3, 3, 4096, 36864, 4, 2, 128, 2, 2, None) == -1            # o aliases part 0, lse does not
+    assert f(o3, l3, 3, 4096, 16384, 4, 2, 128, 2, 1, None) == -1            # aliasing with bf16 output
+    assert "alias" in binding.pec_last_error()

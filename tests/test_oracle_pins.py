@@ -239,6 +239,40 @@ def test_merge_of_disjoint_key_sets_is_attention_over_the_union():
     np.testing.assert_allclose(m[0], ref[0].permute(1, 0, 2).numpy(), atol=1e-12)
 
 
+def test_merge_n_equals_folded_pairwise_merges_and_attention_over_the_union():
+    S, hq, hkv, d = 120, 4, 2, 16
+    q, k, v = _rand((S, hq, d), 171), _rand((S, hkv, d), 172), _rand((S, hkv, d), 173)
+    pos = np.arange(S)
+    sets = [[(0, 10)], [(10, 50), (100, 120)], [(50, 51)], [(51, 100)], [(60, 60)]]   # last one empty
+    parts = [oracle.attn_rows(q, pos, k, v, ivs, True) for ivs in sets]
+    got = oracle.merge_n([p[0] for p in parts], [p[1] for p in parts])
+    acc = parts[0]
+    for part in parts[1:]:
+        acc = oracle.merge(*acc, *part)
+    np.testing.assert_allclose(got[0], acc[0], atol=1e-13)
+    np.testing.assert_allclose(got[1], acc[1], atol=1e-13)
+    full = oracle.attn_rows(q, pos, k, v, [(0, S)], True)
+    np.testing.assert_allclose(got[0], full[0], atol=1e-12)
+    np.testing.assert_allclose(got[1], full[1], atol=1e-12)
+    tq = torch.from_numpy(q).double().permute(1, 0, 2)[None]
+    tk = torch.from_numpy(k).double().repeat_interleave(2, 1).permute(1, 0, 2)[None]
+    tv = torch.from_numpy(v).double().repeat_interleave(2, 1).permute(1, 0, 2)[None]
+    ref = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, is_causal=True)
+    np.testing.assert_allclose(got[0], ref[0].permute(1, 0, 2).numpy(), atol=1e-12)
+
+
+def test_merge_n_closed_form_and_empty_rows():
+    """LSE = ln 1, ln 2, ln 5 -> weights 1/8, 2/8, 5/8, LSE = ln 8 (plain arithmetic); garbage behind
+    an empty part is ignored; all-empty rows give (0, -inf)."""
+    o = [np.full((2, 1, 2), 8.0), np.full((2, 1, 2), 16.0), np.full((2, 1, 2), 1.6), np.full((2, 1, 2), np.nan)]
+    l = [np.array([[0.0], [-np.inf]]), np.array([[math.log(2.0)], [-np.inf]]),
+         np.array([[math.log(5.0)], [-np.inf]]), np.array([[-np.inf], [-np.inf]])]
+    got_o, got_l = oracle.merge_n(o, l)
+    np.testing.assert_allclose(got_o[0], 1.0 + 4.0 + 1.0, atol=1e-14)
+    np.testing.assert_allclose(got_l[0], math.log(8.0), atol=1e-14)
+    assert (got_o[1] == 0).all() and np.isneginf(got_l[1]).all()
+
+
 # ------------------------------------------------------------------ the call-level oracle
 @pytest.mark.parametrize("S,P,align", [(1024, 4, 128), (700, 3, 64), (130, 2, 128), (257, 8, 16)])
 def test_partitions_merged_equal_monolithic(S, P, align):
