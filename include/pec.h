@@ -150,6 +150,46 @@ int pec_attn_merge_n(const void *const *o_parts, const float *const *lse_parts, 
                      int32_t part_dtype, int32_t out_dtype, void *cuda_stream);
 
 /*
+ * Decode attention of a long request's single new token over part of its K/V cache
+ * (Section 5.2: the long request in decode has one query token; its Q is sent to each GPU that
+ * holds part of the K/V, every GPU computes attention over its own part with Eq. 3, and the
+ * partial outputs are merged).  This call is one GPU's share: keys [kv_lo, kv_hi) of
+ * k, v [Tk, Hkv, D] (same layout and strides as pec_prefill_attn; row t = position t), all
+ * visible to the token.  q: device [Hq, D] bf16, head stride q_stride_h elements.  Results:
+ * o [Hq, D] (o_dtype PEC_F32 for a partial to merge, PEC_BF16 for a final output), lse [Hq] fp32,
+ * as defined for pec_prefill_attn; an empty range gives o = 0, lse = -inf.  Two GPUs' results are
+ * combined with pec_attn_merge (rows = 1).
+ *
+ * The key range is cut into num_splits slices (0 = the library chooses) that run in parallel and
+ * leave their partial results in `workspace` (device, 16-byte aligned, at least
+ * pec_decode_workspace_size() bytes, which depends on Hq, the range and num_splits); a second
+ * small kernel combines them.  The workspace contents are scratch: undefined after the call.
+ * `status` as in pec_attn_args, but required.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT,
+ * WORKSPACE, CUDA.
+ */
+typedef struct {
+    const void *q;              /* device; [Hq, D] bf16, 16-byte aligned                        */
+    int64_t q_stride_h;
+    const void *k, *v;          /* device; [Tk, Hkv, D] bf16                                   */
+    int64_t k_stride_t, k_stride_h, v_stride_t, v_stride_h;
+    void *o;                    /* device; [Hq, D] contiguous                                  */
+    int32_t o_dtype;
+    float *lse;                 /* device; [Hq]                                                */
+    int32_t Hq, Hkv, D;         /* D must be 128; Hkv | Hq; Hq / Hkv <= 128                    */
+    int64_t kv_lo, kv_hi;       /* 0 <= kv_lo <= kv_hi <= Tk                                   */
+    int32_t num_splits;         /* 0 = choose; otherwise 1..4096                               */
+    float softmax_scale;        /* 0 selects 1/sqrt(D)                                         */
+    void *workspace;
+    size_t workspace_bytes;
+    int32_t *status;
+} pec_decode_args;
+
+int pec_decode_attn(const pec_decode_args *args, void *cuda_stream);
+
+/* Bytes of workspace pec_decode_attn needs for these arguments (0 if they are invalid). */
+size_t pec_decode_workspace_size(const pec_decode_args *args);
+
+/*
  * Host-side plan of how a request of seq_len tokens is split.  All arrays are
  * host memory owned by the caller; an array pointer may be NULL to skip that
  * output.  Capacities are element counts; the needed counts are always written

@@ -48,6 +48,21 @@ class pec_attn_args(ctypes.Structure):
     ]
 
 
+class pec_decode_args(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("q_stride_h", ctypes.c_int64),
+        ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
+        ("k_stride_t", ctypes.c_int64), ("k_stride_h", ctypes.c_int64),
+        ("v_stride_t", ctypes.c_int64), ("v_stride_h", ctypes.c_int64),
+        ("o", ctypes.c_void_p), ("o_dtype", ctypes.c_int32), ("lse", ctypes.c_void_p),
+        ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("D", ctypes.c_int32),
+        ("kv_lo", ctypes.c_int64), ("kv_hi", ctypes.c_int64),
+        ("num_splits", ctypes.c_int32), ("softmax_scale", ctypes.c_float),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+        ("status", ctypes.c_void_p),
+    ]
+
+
 class pec_plan(ctypes.Structure):
     _fields_ = [
         ("bounds", ctypes.POINTER(ctypes.c_int64)), ("bounds_cap", ctypes.c_int64),
@@ -63,7 +78,7 @@ class pec_plan(ctypes.Structure):
 
 
 EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_attn_merge_n", "pec_plan_partitions",
-           "pec_last_error")
+           "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size")
 PEC_MERGE_MAX_PARTS = 16
 
 
@@ -90,6 +105,10 @@ def load():
     lib.pec_plan_partitions.restype = ctypes.c_int
     lib.pec_plan_partitions.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int64, ctypes.c_int32,
                                         ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(pec_plan)]
+    lib.pec_decode_attn.restype = ctypes.c_int
+    lib.pec_decode_attn.argtypes = [ctypes.POINTER(pec_decode_args), ctypes.c_void_p]
+    lib.pec_decode_workspace_size.restype = ctypes.c_size_t
+    lib.pec_decode_workspace_size.argtypes = [ctypes.POINTER(pec_decode_args)]
     lib.pec_last_error.restype = ctypes.c_char_p
     lib.pec_last_error.argtypes = []
     _lib = lib
@@ -234,6 +253,47 @@ def pec_attn_merge_n(o_parts, lse_parts, *, out_dtype=torch.float32, o_out=None,
     _check(lib.pec_attn_merge_n(op, lp, n, o_out.data_ptr(), lse_out.data_ptr(), rows, Hq, D,
                                 _dtype_code(o_parts[0].dtype), _dtype_code(o_out.dtype), _stream_ptr(stream)))
     return o_out, lse_out
+
+
+def decode_args(q, k, v, o, lse, kv_lo, kv_hi, num_splits=0, softmax_scale=0.0):
+    """Fill a pec_decode_args from tensors (q [Hq,128], k/v [Tk,Hkv,128], o [Hq,128], lse [Hq])."""
+    a = pec_decode_args()
+    a.q, a.q_stride_h = q.data_ptr(), q.stride(0)
+    a.k, a.v = k.data_ptr(), v.data_ptr()
+    a.k_stride_t, a.k_stride_h = k.stride(0), k.stride(1)
+    a.v_stride_t, a.v_stride_h = v.stride(0), v.stride(1)
+    a.o, a.o_dtype, a.lse = o.data_ptr(), _dtype_code(o.dtype), lse.data_ptr()
+    a.Hq, a.Hkv, a.D = q.shape[0], k.shape[1], q.shape[1]
+    a.kv_lo, a.kv_hi = kv_lo, kv_hi
+    a.num_splits, a.softmax_scale = num_splits, float(softmax_scale)
+    a.workspace, a.workspace_bytes = None, 0
+    a.status = status_word(q.device).data_ptr()
+    return a
+
+
+def pec_decode_workspace_size(a) -> int:
+    return int(load().pec_decode_workspace_size(ctypes.byref(a)))
+
+
+def pec_decode_attn(q, k, v, *, kv_lo=0, kv_hi=None, num_splits=0, softmax_scale=0.0, out_dtype=torch.float32,
+                    o=None, lse=None, workspace=None, stream=None):
+    """One GPU's share of a long request's decode step: the new token's attention over keys
+    [kv_lo, kv_hi) of its K/V cache; returns (o [Hq,128], lse [Hq]).  The workspace tensor (uint8,
+    CUDA) is allocated here when not given."""
+    lib = load()
+    assert q.is_cuda and q.dtype == torch.bfloat16 and q.stride(1) == 1 and k.stride(2) == 1 and v.stride(2) == 1
+    kv_hi = k.shape[0] if kv_hi is None else kv_hi
+    if o is None:
+        o = torch.empty((q.shape[0], 128), dtype=out_dtype, device=q.device)
+    if lse is None:
+        lse = torch.empty((q.shape[0],), dtype=torch.float32, device=q.device)
+    a = decode_args(q, k, v, o, lse, kv_lo, kv_hi, num_splits, softmax_scale)
+    need = pec_decode_workspace_size(a)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
+    a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
+    _check(lib.pec_decode_attn(ctypes.byref(a), _stream_ptr(stream)))
+    return o, lse
 
 
 def pec_plan_partitions(seq_len, num_parts, chunk_len=0, align=128, block_m=128, block_n=128,

@@ -96,6 +96,8 @@ static int resolve(const pec_attn_args *a, AttnParams &p)
     p.scale_log2 = (float)((double)p.scale * 1.4426950408889634074);
     p.o_is_bf16 = a->o_dtype == PEC_BF16;
     p.status = a->status;
+    p.splits = 1;
+    p.split_keys = 0;
 
     // Key subset of a single request: zigzag partition cut to the stored K/V prefix.
     int64_t lo[2], hi[2];

@@ -104,6 +104,13 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // An earlier CTA's wait expired: the launch is already lost, leave at once.
         if (p.status && *reinterpret_cast<volatile int32_t *>(p.status) != 0) g.found = 0;
         sh->abort_flag = 0;
+        if (g.found && p.splits > 1) {                        // split-KV launch: this CTA's slice of the keys
+            const int64_t lo = job.iv_lo[0] + (int64_t)blockIdx.z * p.split_keys;
+            const int64_t hi = lo + p.split_keys < job.iv_hi[0] ? lo + p.split_keys : job.iv_hi[0];
+            job.iv_lo[0] = lo;
+            job.iv_hi[0] = hi > lo ? hi : lo;
+            job.out_row0 += (int64_t)blockIdx.z * p.total_rows;
+        }
         if (g.found) {
             g.q_row0 = (int32_t)job.q_row0; g.out_row0 = (int32_t)job.out_row0; g.kv_row0 = (int32_t)job.kv_row0;
             g.cnt[0] = g.cnt[1] = 0;
@@ -460,7 +467,8 @@ int launch_attn_bf16(const AttnParams &p, cudaStream_t stream)
     int64_t tiles = (p.total_rows + kBlockM - 1) / kBlockM;
     if (p.cu_seqlens) tiles += p.B;
     if (tiles > 0x7fffffff || p.Hq > 65535) { set_error("pec_prefill_attn: grid too large"); return PEC_ERR_UNSUPPORTED; }
-    dim3 grid((unsigned)tiles, (unsigned)p.Hq);
+    if (p.splits < 1 || p.splits > 65535) { set_error("pec_prefill_attn: bad split count"); return PEC_ERR_INVALID_ARG; }
+    dim3 grid((unsigned)tiles, (unsigned)p.Hq, (unsigned)p.splits);
     attn_bf16_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, p);
     const cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("pec_prefill_attn: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }

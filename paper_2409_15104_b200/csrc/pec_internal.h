@@ -29,6 +29,10 @@ struct AttnParams {
     float scale_log2;                // scale * log2(e)
     int32_t o_is_bf16;
     int32_t *status;
+    // Split-KV launches (decode): grid.z CTAs each take `split_keys` keys of interval 0 and write
+    // their partial to slice blockIdx.z of o / lse ([splits][total_rows][Hq][D] / [splits][total_rows][Hq]).
+    int32_t splits;                  // 1 = ordinary launch
+    int64_t split_keys;              // multiple of 128
 };
 
 void set_error(const char *fmt, ...);
@@ -43,6 +47,13 @@ int launch_attn_bf16(const AttnParams &p, cudaStream_t stream);
 int launch_merge(const float *o_a, const float *lse_a, const float *o_b, const float *lse_b,
                  void *o_out, float *lse_out, int64_t items, int out_is_bf16, int inplace,
                  cudaStream_t stream);
+
+// Split-KV decode (pec_decode.cu): sizes of the scratch one call needs.
+struct DecodeShape {
+    int32_t splits;
+    int64_t split_keys;
+    size_t scratch_bytes;            // partial O + partial LSE of every split
+};
 
 struct MergeParts {
     const float *o[PEC_MERGE_MAX_PARTS];

@@ -207,3 +207,38 @@ def test_canaries_around_outputs_stay_untouched(pec):
     pec.check_status()
     assert (obuf[:pad] == 7).all() and (obuf[pad + S:] == 7).all()
     assert (lbuf[:pad] == 7).all() and (lbuf[pad + S:] == 7).all()
+
+
+# ------------------------------------------------------------------ split-KV decode of a long request
+@pytest.mark.parametrize("L,hq,hkv,lo,hi,splits", [
+    (1, 4, 2, 0, 1, 0), (127, 8, 8, 0, 127, 0), (1000, 32, 8, 0, 1000, 0), (5000, 32, 8, 1234, 4999, 0),
+    (4096, 64, 8, 0, 4096, 7), (3000, 16, 2, 0, 3000, 1), (777, 8, 2, 300, 300, 0), (20000, 32, 8, 0, 20000, 0),
+])
+@pytest.mark.parametrize("out", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_decode_split_kv(pec, L, hq, hkv, lo, hi, splits, out):
+    _, k, v = _qkv(11000 + L, L, hq, hkv, torch.bfloat16)
+    q = workloads.normal_tensor(11001 + L, 1, (1, hq, 128), torch.bfloat16)
+    want = oracle.attn_rows(q, [L - 1], k, v, [(lo, hi)] if hi > lo else [], False)
+    dq, dk, dv = _gpu(q[0], k, v)
+    o, lse = pec.pec_decode_attn(dq, dk, dv, kv_lo=lo, kv_hi=hi, num_splits=splits, out_dtype=out)
+    pec.check_status()
+    compare(o[None], lse[None], *want, 2e-2, 1e-3, f"decode L={L} [{lo},{hi}) splits={splits}")
+
+
+def test_decode_on_two_kv_halves_merges_to_the_whole(pec):
+    """The colocation example: the long request's K/V split over two holders, partial outputs merged."""
+    L, hq, hkv = 6000, 32, 8
+    _, k, v = _qkv(12000, L, hq, hkv, torch.bfloat16)
+    q = workloads.normal_tensor(12001, 1, (1, hq, 128), torch.bfloat16)
+    dq, dk, dv = _gpu(q[0], k, v)
+    a = pec.pec_decode_attn(dq, dk, dv, kv_lo=0, kv_hi=3100)
+    b = pec.pec_decode_attn(dq, dk, dv, kv_lo=3100, kv_hi=L)
+    o, lse = pec.pec_attn_merge(a[0][None], a[1][None], b[0][None], b[1][None], out_dtype=torch.bfloat16)
+    pec.check_status()
+    want = oracle.attn_rows(q, [L - 1], k, v, [(0, L)], False)
+    compare(o, lse, *want, 2e-2, 1e-3, "decode halves merged")
+    # decode of the last token equals the last row of a causal prefill of the same request
+    qfull = torch.cat([workloads.normal_tensor(12002, 1, (L - 1, hq, 128), torch.bfloat16), q])
+    po, pl = pec.pec_prefill_attn(qfull.to(DEV), dk, dv, chunk_start=L - 1, chunk_len=1, seq_len=L)
+    pec.check_status()
+    compare(po, pl, *want, 2e-2, 1e-3, "prefill last row")

@@ -130,3 +130,27 @@ def test_merge_n_validates_on_the_host():
     assert f(o3, l3, 3, 4096, 36864, 4, 2, 128, 2, 2, None) == -1            # o aliases part 0, lse does not
     assert f(o3, l3, 3, 4096, 16384, 4, 2, 128, 2, 1, None) == -1            # aliasing with bf16 output
     assert "alias" in binding.pec_last_error()
+
+
+def test_decode_validates_on_the_host_and_sizes_its_workspace():
+    lib = binding.load()
+    a = binding.pec_decode_args()
+    a.q = a.k = a.v = a.o = a.lse = a.status = 4096
+    a.q_stride_h = 128
+    a.k_stride_t = a.v_stride_t = 8 * 128
+    a.k_stride_h = a.v_stride_h = 128
+    a.o_dtype, a.Hq, a.Hkv, a.D = binding.PEC_F32, 32, 8, 128
+    a.kv_lo, a.kv_hi, a.num_splits = 0, 100000, 10
+    need = lib.pec_decode_workspace_size(ctypes.byref(a))
+    # 10 slices of ceil(10000/128)*128 = 10112 keys -> still 10 slices; 516 bytes per (slice, head)
+    assert need == 10 * 32 * 516
+    assert lib.pec_decode_attn(ctypes.byref(a), None) == -4            # no workspace given
+    a.workspace, a.workspace_bytes = 4096, need - 1
+    assert lib.pec_decode_attn(ctypes.byref(a), None) == -4
+    for field, val, code in [("D", 64, -2), ("Hq", 30, -1), ("kv_hi", -1, -1), ("num_splits", 5000, -1),
+                             ("q", 4100, -3), ("k_stride_t", 1028, -3), ("status", None, -1), ("o_dtype", 9, -2)]:
+        old = getattr(a, field)
+        setattr(a, field, val)
+        assert lib.pec_decode_attn(ctypes.byref(a), None) == code, field
+        assert lib.pec_decode_workspace_size(ctypes.byref(a)) == 0
+        setattr(a, field, old)
