@@ -190,6 +190,36 @@ int pec_decode_attn(const pec_decode_args *args, void *cuda_stream);
 size_t pec_decode_workspace_size(const pec_decode_args *args);
 
 /*
+ * pec_decode_attn without a workspace argument.  (The paper has no counterpart for this call; it
+ * exists for the way such a kernel gets deployed.)
+ *
+ * Who needs it: a serving engine of the kind the paper builds on hands every free byte of HBM
+ * to its KV-cache pool at start-up, and the decode step of a colocated long request is issued
+ * from a scheduler loop that must not stall.  Such a caller cannot ask the driver for memory at
+ * that point: cudaMalloc may simply fail because nothing is left, and even when it succeeds it
+ * synchronises the whole device, which is exactly the pause the scheduler is trying to avoid.
+ * Nor may the call be handed a slice of the engine's pool by a layer that does not own it.
+ *
+ * So this variant keeps its scratch inside the library: a fixed array of
+ * PEC_DECODE_STATIC_SCRATCH_BYTES in device memory that every GPU loading the library carries
+ * from load until the process exits.  It performs no allocation and frees nothing.  Arguments
+ * and results are those of pec_decode_attn, except that `workspace` and `workspace_bytes` are
+ * ignored.  A call whose slices need more scratch than the array holds (slices x Hq x 516
+ * bytes; see pec_decode_workspace_size) is refused with PEC_ERR_WORKSPACE and a message that
+ * names both sizes: lower num_splits, or use pec_decode_attn.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current) and remembers it; make that first call outside any stream capture.  All calls on a
+ * device share the one array and it keeps whatever the previous call left there.  Nothing in
+ * it has to start at zero - each call overwrites every partial it later reads - but two calls
+ * that overlap on the GPU (different streams, or one stream replayed concurrently) would
+ * overwrite each other's partials: keep them ordered.
+ * Errors: as pec_decode_attn, plus PEC_ERR_CUDA if the address lookup fails.
+ */
+#define PEC_DECODE_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+int pec_decode_attn_static(const pec_decode_args *args, void *cuda_stream);
+
+/*
  * Host-side plan of how a request of seq_len tokens is split.  All arrays are
  * host memory owned by the caller; an array pointer may be NULL to skip that
  * output.  Capacities are element counts; the needed counts are always written

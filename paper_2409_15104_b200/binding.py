@@ -78,7 +78,8 @@ class pec_plan(ctypes.Structure):
 
 
 EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_attn_merge_n", "pec_plan_partitions",
-           "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size")
+           "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size", "pec_decode_attn_static")
+PEC_DECODE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 PEC_MERGE_MAX_PARTS = 16
 
 
@@ -107,6 +108,8 @@ def load():
                                         ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(pec_plan)]
     lib.pec_decode_attn.restype = ctypes.c_int
     lib.pec_decode_attn.argtypes = [ctypes.POINTER(pec_decode_args), ctypes.c_void_p]
+    lib.pec_decode_attn_static.restype = ctypes.c_int
+    lib.pec_decode_attn_static.argtypes = [ctypes.POINTER(pec_decode_args), ctypes.c_void_p]
     lib.pec_decode_workspace_size.restype = ctypes.c_size_t
     lib.pec_decode_workspace_size.argtypes = [ctypes.POINTER(pec_decode_args)]
     lib.pec_last_error.restype = ctypes.c_char_p

@@ -9,6 +9,7 @@
 // go to scratch memory and are combined by the small kernel below (same LSE merge as pec_attn_merge).
 #include <cuda_bf16.h>
 #include <cmath>
+#include <mutex>
 #include "pec_internal.h"
 
 namespace pec {
@@ -132,9 +133,56 @@ static int run_decode(const pec_decode_args *a, const DecodeShape &shape, void *
     return PEC_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Built-in scratch for pec_decode_attn_static.  The array lives in every GPU that loads the
+// library, from load to exit.  Its name is only a handle on the host side: the device address
+// is looked up once per device with cudaGetSymbolAddress and cached here.
+static __device__ __align__(256) unsigned char g_decode_scratch[PEC_DECODE_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_scratch_mutex;
+static void *g_scratch_ptr[kMaxDevices] = {};
+
+// Device address of the built-in scratch on the current device (nullptr + error text on failure).
+static void *static_scratch_for_current_device(const char *who)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        set_error("%s: cannot identify the current device", who);
+        return nullptr;
+    }
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_ptr[dev]) {
+        void *ptr = nullptr;
+        const cudaError_t err = cudaGetSymbolAddress(&ptr, g_decode_scratch);
+        if (err != cudaSuccess || !ptr) {
+            set_error("%s: cudaGetSymbolAddress failed on device %d: %s", who, dev, cudaGetErrorString(err));
+            return nullptr;
+        }
+        g_scratch_ptr[dev] = ptr;
+    }
+    return g_scratch_ptr[dev];
+}
+
 }  // namespace pec
 
 using namespace pec;
+
+extern "C" int pec_decode_attn_static(const pec_decode_args *args, void *cuda_stream)
+{
+    DecodeShape shape;
+    const int rc = check_decode(args, shape, "pec_decode_attn_static");
+    if (rc != PEC_OK) return rc;
+    if (shape.scratch_bytes > (size_t)PEC_DECODE_STATIC_SCRATCH_BYTES) {
+        set_error("pec_decode_attn_static: this call needs %zu bytes of scratch (slices x Hq x 516) but the built-in "
+                  "scratch holds %d; pass a smaller num_splits or use pec_decode_attn with a workspace",
+                  shape.scratch_bytes, PEC_DECODE_STATIC_SCRATCH_BYTES);
+        return PEC_ERR_WORKSPACE;
+    }
+    void *scratch = static_scratch_for_current_device("pec_decode_attn_static");
+    if (!scratch) return PEC_ERR_CUDA;
+    return run_decode(args, shape, scratch, static_cast<cudaStream_t>(cuda_stream), "pec_decode_attn_static");
+}
 
 extern "C" size_t pec_decode_workspace_size(const pec_decode_args *args)
 {
