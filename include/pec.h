@@ -251,6 +251,36 @@ typedef struct {
 int pec_plan_partitions(int64_t seq_len, int32_t num_parts, int64_t chunk_len, int32_t align,
                         int32_t block_m, int32_t block_n, int32_t causal, pec_plan *plan);
 
+/*
+ * Intra-node SP strategy selection for a long prefill (Section 5.3).  With TP size T, G GPUs per
+ * node, per-GPU segment length s, model width d, N_h query heads and N_kv KV heads of size d_h, the
+ * paper gives, per stage and strategy, the communication volume in a node and the computation
+ * volume on a GPU:
+ *   attention stage, Megatron SP: comm 2sd(T-1)G            comp 2sd(N_h+N_kv)d_h/T + 4(sT)^2 d/T + 2sd^2
+ *   attention stage, Ulysses SP : comm 2s(N_h+N_kv)d_h(G-1) + (d(N_h+N_kv)d_h + d^2)G(T-1)/T
+ *                                 comp 2sd(N_h+N_kv)d_h + 4(sG)^2 d/G + 2sd^2
+ *   MLP stage, Megatron SP      : comm 2sd(T-1)G            comp 16sd^2
+ *   MLP stage, Ulysses SP       : comm 8d^2(T-1)G/T         comp 16sd^2
+ * and picks, among the four combinations, the one with the lowest estimated latency.  The paper
+ * does not say how volumes become time; this library's reading: seconds = comm elements *
+ * elem_bytes / node_bw + comp / gpu_flops, summed over the two stages.  Host arithmetic in
+ * double; ties go to the lower index (Megatron before Ulysses).  Strategy codes: 0 = Megatron SP,
+ * 1 = Ulysses SP.  comm[stage][strategy] and comp[stage][strategy] (stage 0 = attention,
+ * 1 = MLP) return the volumes, seconds[2*attn + mlp] the four estimates.
+ * Errors: INVALID_ARG (NULL, non-positive sizes, T or G below 1, non-positive rates).
+ */
+typedef struct {
+    double s, d, n_h, n_kv, d_h, T, G;
+    double elem_bytes;          /* bytes per communicated element (2 for bf16)                  */
+    double node_bw;             /* bytes per second the node moves in total                     */
+    double gpu_flops;           /* operations per second of one GPU                             */
+} pec_sp_inputs;
+typedef struct {
+    int32_t attn_strategy, mlp_strategy;
+    double comm[2][2], comp[2][2], seconds[4];
+} pec_sp_choice;
+int pec_select_sp(const pec_sp_inputs *in, pec_sp_choice *out);
+
 /* Text describing the last non-zero return on this thread (never NULL). */
 const char *pec_last_error(void);
 

@@ -9,6 +9,8 @@ from .reference import (  # noqa: F401
     varlen_attn,
     merge,
     merge_n,
+    sp_volumes,
+    select_sp,
     plan_partitions,
     partition_intervals,
     oracle_threads,

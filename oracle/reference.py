@@ -239,3 +239,41 @@ def merge_n(o_parts, lse_parts):
         c = np.where(empty, 0.0, w[i] / np.where(empty, 1.0, tot))
         o += c[..., None] * np.where(c[..., None] == 0.0, 0.0, oi)
     return o, lse
+
+
+# --------------------------------------------------------------------------- SP strategy cost model
+def sp_volumes(s, d, n_h, n_kv, d_h, T, G):
+    """Section 5.3's communication (per node) and computation (per GPU) volumes, written term by term
+    with exact rational arithmetic: {(stage, strategy): (comm, comp)} for stage in ("attn", "mlp") and
+    strategy in ("megatron", "ulysses")."""
+    from fractions import Fraction as F
+    s, d, n_h, n_kv, d_h, T, G = (F(x) for x in (s, d, n_h, n_kv, d_h, T, G))
+    qkv = 2 * s * d * (n_h + n_kv) * d_h          # QKV generation on a full segment
+    out_proj = 2 * s * d * d                      # post-self-attention linear
+    vols = {}
+    # attention stage, Megatron SP: all-gather + reduce-scatter; QKV split over T, attention over s*T tokens / T
+    vols[("attn", "megatron")] = (2 * s * d * (T - 1) * G, qkv / T + 4 * (s * T) ** 2 * d / T + out_proj)
+    # attention stage, Ulysses SP: two all-to-alls + parameter transfer; attention over s*G tokens / G
+    a2a = 2 * s * (n_h + n_kv) * d_h * (G - 1)
+    params = (d * (n_h + n_kv) * d_h + d * d) * G * (T - 1) / T
+    vols[("attn", "ulysses")] = (a2a + params, qkv + 4 * (s * G) ** 2 * d / G + out_proj)
+    # MLP stage: 16 s d^2 either way; Megatron moves embeddings, Ulysses moves the 8 d^2 parameters
+    vols[("mlp", "megatron")] = (2 * s * d * (T - 1) * G, 16 * s * d * d)
+    vols[("mlp", "ulysses")] = (8 * d * d * (T - 1) * G / T, 16 * s * d * d)
+    return vols
+
+
+def select_sp(s, d, n_h, n_kv, d_h, T, G, elem_bytes, node_bw, gpu_flops):
+    """The combination with the lowest estimated latency (comm bytes / node_bw + comp / gpu_flops);
+    ties go to Megatron.  Returns ((attn, mlp), {combo: seconds})."""
+    from fractions import Fraction as F
+    vols = sp_volumes(s, d, n_h, n_kv, d_h, T, G)
+    times = {}
+    for a in ("megatron", "ulysses"):
+        for m in ("megatron", "ulysses"):
+            comm = vols[("attn", a)][0] + vols[("mlp", m)][0]
+            comp = vols[("attn", a)][1] + vols[("mlp", m)][1]
+            times[(a, m)] = comm * F(elem_bytes) / F(node_bw) + comp / F(gpu_flops)
+    order = [("megatron", "megatron"), ("megatron", "ulysses"), ("ulysses", "megatron"), ("ulysses", "ulysses")]
+    best = min(order, key=lambda c: (times[c], order.index(c)))
+    return best, times

@@ -63,6 +63,15 @@ class pec_decode_args(ctypes.Structure):
     ]
 
 
+class pec_sp_inputs(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_double) for n in ("s", "d", "n_h", "n_kv", "d_h", "T", "G", "elem_bytes", "node_bw", "gpu_flops")]
+
+
+class pec_sp_choice(ctypes.Structure):
+    _fields_ = [("attn_strategy", ctypes.c_int32), ("mlp_strategy", ctypes.c_int32),
+                ("comm", (ctypes.c_double * 2) * 2), ("comp", (ctypes.c_double * 2) * 2), ("seconds", ctypes.c_double * 4)]
+
+
 class pec_plan(ctypes.Structure):
     _fields_ = [
         ("bounds", ctypes.POINTER(ctypes.c_int64)), ("bounds_cap", ctypes.c_int64),
@@ -78,7 +87,7 @@ class pec_plan(ctypes.Structure):
 
 
 EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_attn_merge_n", "pec_plan_partitions",
-           "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size", "pec_decode_attn_static")
+           "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size", "pec_decode_attn_static", "pec_select_sp")
 PEC_DECODE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 PEC_MERGE_MAX_PARTS = 16
 
@@ -112,6 +121,8 @@ def load():
     lib.pec_decode_attn_static.argtypes = [ctypes.POINTER(pec_decode_args), ctypes.c_void_p]
     lib.pec_decode_workspace_size.restype = ctypes.c_size_t
     lib.pec_decode_workspace_size.argtypes = [ctypes.POINTER(pec_decode_args)]
+    lib.pec_select_sp.restype = ctypes.c_int
+    lib.pec_select_sp.argtypes = [ctypes.POINTER(pec_sp_inputs), ctypes.POINTER(pec_sp_choice)]
     lib.pec_last_error.restype = ctypes.c_char_p
     lib.pec_last_error.argtypes = []
     _lib = lib
@@ -297,6 +308,18 @@ def pec_decode_attn(q, k, v, *, kv_lo=0, kv_hi=None, num_splits=0, softmax_scale
     a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
     _check(lib.pec_decode_attn(ctypes.byref(a), _stream_ptr(stream)))
     return o, lse
+
+
+def pec_select_sp(s, d, n_h, n_kv, d_h, T, G, elem_bytes=2.0, node_bw=1.0, gpu_flops=1.0):
+    """Section 5.3's strategy choice; returns a dict (strategies: 0 = Megatron SP, 1 = Ulysses SP)."""
+    lib = load()
+    i = pec_sp_inputs(s, d, n_h, n_kv, d_h, T, G, elem_bytes, node_bw, gpu_flops)
+    o = pec_sp_choice()
+    _check(lib.pec_select_sp(ctypes.byref(i), ctypes.byref(o)))
+    return {"attn_strategy": o.attn_strategy, "mlp_strategy": o.mlp_strategy,
+            "comm": [[o.comm[a][b] for b in range(2)] for a in range(2)],
+            "comp": [[o.comp[a][b] for b in range(2)] for a in range(2)],
+            "seconds": [o.seconds[i] for i in range(4)]}
 
 
 def pec_plan_partitions(seq_len, num_parts, chunk_len=0, align=128, block_m=128, block_n=128,

@@ -105,3 +105,34 @@ extern "C" int pec_plan_partitions(int64_t seq_len, int32_t num_parts, int64_t c
     }
     return PEC_OK;
 }
+
+// Section 5.3's closed forms for the hybrid SP strategy choice (host arithmetic only).
+extern "C" int pec_select_sp(const pec_sp_inputs *in, pec_sp_choice *out)
+{
+    if (!in || !out) { set_error("pec_select_sp: NULL argument"); return PEC_ERR_INVALID_ARG; }
+    const double s = in->s, d = in->d, nh = in->n_h, nkv = in->n_kv, dh = in->d_h, T = in->T, G = in->G;
+    if (!(s > 0 && d > 0 && nh > 0 && nkv > 0 && dh > 0 && T >= 1 && G >= 1 && in->elem_bytes > 0 && in->node_bw > 0 && in->gpu_flops > 0)) {
+        set_error("pec_select_sp: sizes and rates must be positive, T and G at least 1");
+        return PEC_ERR_INVALID_ARG;
+    }
+    const double heads = (nh + nkv) * dh;
+    out->comm[0][0] = 2 * s * d * (T - 1) * G;
+    out->comp[0][0] = 2 * s * d * heads / T + 4 * (s * T) * (s * T) * d / T + 2 * s * d * d;
+    out->comm[0][1] = 2 * s * heads * (G - 1) + (d * heads + d * d) * G * (T - 1) / T;
+    out->comp[0][1] = 2 * s * d * heads + 4 * (s * G) * (s * G) * d / G + 2 * s * d * d;
+    out->comm[1][0] = 2 * s * d * (T - 1) * G;
+    out->comp[1][0] = 16 * s * d * d;
+    out->comm[1][1] = 8 * d * d * (T - 1) * G / T;
+    out->comp[1][1] = 16 * s * d * d;
+    int best = 0;
+    for (int a = 0; a < 2; ++a)
+        for (int m = 0; m < 2; ++m) {
+            const double t = (out->comm[0][a] + out->comm[1][m]) * in->elem_bytes / in->node_bw +
+                             (out->comp[0][a] + out->comp[1][m]) / in->gpu_flops;
+            out->seconds[2 * a + m] = t;
+            if (t < out->seconds[best]) best = 2 * a + m;
+        }
+    out->attn_strategy = best >> 1;
+    out->mlp_strategy = best & 1;
+    return PEC_OK;
+}
