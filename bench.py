@@ -353,13 +353,112 @@ def run_decode(args):
                       "max_abs_err_vs_oracle": err}), flush=True)
 
 
+def _short_batch(wl, dev, seed_offset=0):
+    lens = workloads.short_lengths(wl.seed, wl.short_batch)
+    cu = workloads.cu_seqlens(lens)
+    q, k, v = workloads.qkv(wl.seed + 100 + seed_offset, cu[-1], wl.hq, wl.hkv, 128, wl.dtype)
+    pairs = sum(workloads.causal_pairs(n) for n in lens)
+    return (q.to(dev), k.to(dev), v.to(dev), torch.tensor(cu, dtype=torch.int32, device=dev), cu[-1], pairs)
+
+
+def run_short_batch(args, wl):
+    """Extra line: the packed short-request batch (c2) alone."""
+    from paper_2409_15104_b200 import binding
+    from paper_2409_15104_b200.prefill import varlen_prefill
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    q, k, v, cu, T, pairs = _short_batch(wl, dev)
+    o = torch.empty((T, wl.hq, 128), dtype=wl.dtype, device=dev)
+    lse = torch.empty((T, wl.hq), dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    for _ in range(max(args.warmup, 3)):
+        varlen_prefill(q, k, v, cu, o=o, lse=lse)
+    torch.cuda.synchronize()
+    evs = []
+    for _ in range(min(args.steps, 50)):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); varlen_prefill(q, k, v, cu, o=o, lse=lse); e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    binding.check_status()
+    ms = statistics.median(a.elapsed_time(b) for a, b in evs)
+    fl = workloads.attention_flops(pairs, wl.hq)
+    print(json.dumps({"metric": "short-request varlen batch, attention TFLOP/s (extra line, not the headline)",
+                      "value": fl / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms, "n_gpus": 1, "dtype": "bf16",
+                      "data": "synthetic", "tokens_per_s": T / (ms * 1e-3),
+                      "config": {"workload": f"{wl.name}: {wl.note}", "requests": wl.short_batch, "tokens": T,
+                                 "pairs_per_head": pairs, "l2": "256 MiB written between timed calls"}}), flush=True)
+
+
+def run_preempted(args, wl):
+    """Extra line: c4 - a long prefill as 16 resumed chunks on a low-priority stream with a short-request
+    batch arriving on a high-priority stream while chunk 4 runs."""
+    from paper_2409_15104_b200 import binding
+    from paper_2409_15104_b200.prefill import chunked_prefill, varlen_prefill
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    S, C = wl.seq_len, wl.chunk_len
+    q, k, v = (t.to(dev) for t in workloads.qkv(wl.seed, S, wl.hq, wl.hkv, 128, wl.dtype))
+    sq, sk, sv, cu, T, spairs = _short_batch(wl, dev)
+    o = torch.empty((S, wl.hq, 128), dtype=wl.dtype, device=dev)
+    lse = torch.empty((S, wl.hq), dtype=torch.float32, device=dev)
+    so = torch.empty((T, wl.hq, 128), dtype=wl.dtype, device=dev)
+    sl = torch.empty((T, wl.hq), dtype=torch.float32, device=dev)
+    lo, hi = torch.cuda.Stream(priority=0), torch.cuda.Stream(priority=-1)
+
+    def timed(fn):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter(); fn(); torch.cuda.synchronize()
+        return (time.perf_counter() - t0) * 1e3
+
+    def long_only():
+        chunked_prefill(q, k, v, C, o, lse, stream=lo)
+
+    def short_only():
+        varlen_prefill(sq, sk, sv, cu, o=so, lse=sl, stream=hi)
+
+    marks = {}
+
+    def both():
+        def arrive(c):
+            if c == 3:                                         # the batch arrives once chunk 3 has finished
+                ev = torch.cuda.Event(enable_timing=True); ev.record(lo)
+                hi.wait_event(ev)
+                s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                s0.record(hi); short_only(); s1.record(hi)
+                marks["short"] = (s0, s1)
+        chunked_prefill(q, k, v, C, o, lse, stream=lo, between_chunks=arrive)
+
+    for fn in (long_only, short_only, both):
+        timed(fn)                                              # warm-up
+    reps = 3
+    t_long = min(timed(long_only) for _ in range(reps))
+    t_short = min(timed(short_only) for _ in range(reps))
+    t_both, lat = [], []
+    for _ in range(reps):
+        t_both.append(timed(both))
+        lat.append(marks["short"][0].elapsed_time(marks["short"][1]))
+    binding.check_status()
+    fl_long = workloads.attention_flops(workloads.causal_pairs(S), wl.hq)
+    fl_short = workloads.attention_flops(spairs, wl.hq)
+    print(json.dumps({"metric": "preempted long prefill with a colocated short batch (extra line, not the headline)",
+                      "value": (fl_long + fl_short) / (min(t_both) * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": 1,
+                      "dtype": "bf16", "data": "synthetic",
+                      "long_alone_ms": t_long, "long_alone_tflops": fl_long / (t_long * 1e-3) / 1e12,
+                      "short_alone_ms": t_short, "interleaved_ms": min(t_both),
+                      "short_batch_latency_when_colocated_ms": min(lat), "short_batch_latency_worst_ms": max(lat),
+                      "timing": "host wall clock around a synchronised region (multi-stream); short latency by CUDA events",
+                      "config": {"workload": f"{wl.name}: {wl.note}", "chunks": S // C, "short_tokens": T}}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["c3", "c5", "decode"], default="c3")
+    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode"], default="c3")
     ap.add_argument("--reference-seconds", type=float, default=0.0,
                     help="--impl reference: CPU seconds per step (default: 90 s spread over the steps, 2-20 s each)")
     ap.add_argument("--profile", action="store_true",
@@ -370,6 +469,12 @@ def main():
         run_decode(args)
         return
     wl = workloads.WORKLOADS[args.workload]
+    if args.workload == "c2":
+        run_short_batch(args, wl)
+        return
+    if args.workload == "c4":
+        run_preempted(args, wl)
+        return
     if args.impl == "reference":
         run_reference(args, wl)
     else:
