@@ -17,6 +17,7 @@ def compare(o_gpu, lse_gpu, o_ref, lse_ref, tol_o, tol_lse, what=""):
     err_o = float(np.abs(o - o_ref).max()) if o.size else 0.0
     fin = ~empty
     err_l = float(np.abs(lse[fin] - lse_ref[fin]).max()) if fin.any() else 0.0
+    print(f"[parity] {what}: max|dO| = {err_o:.3e} (tol {tol_o:g}), max|dLSE| = {err_l:.3e} (tol {tol_lse:g})")
     assert err_o <= tol_o, f"{what}: max |dO| = {err_o:.3e} > {tol_o}"
     assert err_l <= tol_lse, f"{what}: max |dLSE| = {err_l:.3e} > {tol_lse}"
     return err_o, err_l
