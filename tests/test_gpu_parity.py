@@ -242,3 +242,45 @@ def test_decode_on_two_kv_halves_merges_to_the_whole(pec):
     po, pl = pec.pec_prefill_attn(qfull.to(DEV), dk, dv, chunk_start=L - 1, chunk_len=1, seq_len=L)
     pec.check_status()
     compare(po, pl, *want, 2e-2, 1e-3, "prefill last row")
+
+
+# ------------------------------------------------------------------ the calls enqueue only: CUDA-graph capture
+def test_partitioned_step_can_be_captured_and_replayed(pec):
+    """No call allocates or synchronises, so a whole step (8 partials + n-way merge) captures into a CUDA
+    graph; replays on new inputs match the eager result bit for bit."""
+    from paper_2409_15104_b200.prefill import PartitionedPrefill
+    S, hq, hkv, P = 2048, 8, 2, 4
+    q, k, v = _gpu(*_qkv(13000, S, hq, hkv, torch.bfloat16))
+    runner = PartitionedPrefill(S, hq, P, torch.bfloat16, DEV)
+    o_eager, l_eager = (t.clone() for t in runner.run(q, k, v))       # also the warm-up outside capture
+    pec.check_status()
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            runner.run(q, k, v, stream=stream)
+    runner.out_o.zero_(); runner.out_l.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(runner.out_o, o_eager) and torch.equal(runner.out_l, l_eager)
+    q2, k2, v2 = _gpu(*_qkv(13001, S, hq, hkv, torch.bfloat16))
+    q.copy_(q2); k.copy_(k2); v.copy_(v2)                              # same buffers, new contents
+    graph.replay()
+    torch.cuda.synchronize()
+    pec.check_status()
+    want = oracle.prefill_attn(q2.cpu(), k2.cpu(), v2.cpu(), seq_len=S)
+    compare(runner.out_o, runner.out_l, *want, 2e-2, 1e-3, "graph replay")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_non_causal_partition_of_a_chunk(pec, dtype):
+    S, P, c0, n = 900, 3, 256, 300
+    q, k, v = _qkv(14000, S, 4, 2, dtype)
+    for p in range(P):
+        want = oracle.prefill_attn(q, k, v, seq_len=S, chunk_start=c0, chunk_len=n, kv_len=700, part_id=p,
+                                   num_parts=P, part_align=32, causal=False)
+        o, lse = pec.pec_prefill_attn(*_gpu(q, k, v), seq_len=S, chunk_start=c0, chunk_len=n, kv_len=700, part_id=p,
+                                      num_parts=P, part_align=32, causal=False)
+        pec.check_status()
+        compare(o, lse, *want, *TOL[dtype], f"non-causal chunk x partition {p}")
