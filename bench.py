@@ -116,7 +116,7 @@ def run_reference(args, wl):
     if rank != 0:
         return
     q, k, v = workloads.qkv(wl.seed, wl.seq_len, wl.hq, wl.hkv, 128, wl.dtype)
-    per_step = args.reference_seconds or max(2.0, min(20.0, 90.0 / (args.steps + args.warmup)))
+    per_step = args.reference_seconds or max(0.15, min(20.0, 90.0 / (args.steps + args.warmup)))   # ~90 s in all
     for _ in range(args.warmup):
         oracle_sample(wl, q, k, v, target_s=per_step)
     res = [oracle_sample(wl, q, k, v, target_s=per_step) for _ in range(args.steps)]
@@ -460,7 +460,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode"], default="c3")
     ap.add_argument("--reference-seconds", type=float, default=0.0,
-                    help="--impl reference: CPU seconds per step (default: 90 s spread over the steps, 2-20 s each)")
+                    help="--impl reference: CPU seconds per step (default: 90 s spread over the steps, 0.15-20 s each)")
     ap.add_argument("--profile", action="store_true",
                     help="profiling runs: skip the end-to-end and CPU-baseline legs (the printed line is not a result)")
     args = ap.parse_args()
