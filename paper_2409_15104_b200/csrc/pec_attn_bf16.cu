@@ -52,7 +52,13 @@ struct Geom {
     int32_t n[2];                // key tiles each stage takes part in (a prefix of the CTA's walk)
     int32_t lo[2], hi[2];        // visible-key intervals (positions)
     int32_t cnt[2];              // key tiles per interval walked by the CTA (union over both stages)
-    int32_t n_max;               // cnt[0] + cnt[1]
+    int32_t n_max;               // cnt[0] + cnt[1] (dual: the larger of the two stages' counts)
+    // Split-KV (decode) launches run "dual": both stages hold the same query rows and each takes its
+    // own key slice (interval st belongs to stage st), so a CTA keeps two slices in flight and one
+    // slice's softmax overlaps the other's MMAs.
+    int32_t dual;
+    int32_t q_st_stride;         // query-row distance between the stages (128, or 0 when dual)
+    int32_t out_st_stride;       // output-row distance between the stages (128, or rows per slice when dual)
 };
 
 struct Shared {
@@ -104,14 +110,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // An earlier CTA's wait expired: the launch is already lost, leave at once.
         if (p.status && *reinterpret_cast<volatile int32_t *>(p.status) != 0) g.found = 0;
         sh->abort_flag = 0;
-        if (g.found && p.splits > 1) {                        // split-KV launch: this CTA's slice of the keys
-            const int64_t lo = job.iv_lo[0] + (int64_t)blockIdx.z * p.split_keys;
-            const int64_t hi = lo + p.split_keys < job.iv_hi[0] ? lo + p.split_keys : job.iv_hi[0];
-            job.iv_lo[0] = lo;
-            job.iv_hi[0] = hi > lo ? hi : lo;
-            job.out_row0 += (int64_t)blockIdx.z * p.total_rows;
-        }
-        if (g.found) {
+        g.dual = (p.splits > 1) ? 1 : 0;
+        g.q_st_stride = kTile;
+        g.out_st_stride = kTile;
+        if (g.found && !g.dual) {
             g.q_row0 = (int32_t)job.q_row0; g.out_row0 = (int32_t)job.out_row0; g.kv_row0 = (int32_t)job.kv_row0;
             g.cnt[0] = g.cnt[1] = 0;
             for (int t = 0; t < 2; ++t) { g.lo[t] = (int32_t)job.iv_lo[t]; g.hi[t] = (int32_t)job.iv_hi[t]; }
@@ -133,6 +135,28 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 }
             }
             g.n_max = g.cnt[0] + g.cnt[1];
+        }
+        if (g.found && g.dual) {                              // stage st takes key slice 2 * blockIdx.z + st
+            g.q_row0 = (int32_t)job.q_row0; g.kv_row0 = (int32_t)job.kv_row0;
+            g.q_st_stride = 0;
+            g.out_st_stride = (int32_t)p.total_rows;
+            g.out_row0 = (int32_t)job.out_row0 + 2 * (int32_t)blockIdx.z * (int32_t)p.total_rows;
+            g.n_max = 0;
+            for (int st = 0; st < 2; ++st) {
+                const int64_t slice = 2 * (int64_t)blockIdx.z + st;
+                int64_t lo = job.iv_lo[0] + slice * p.split_keys;
+                int64_t hi = lo + p.split_keys < job.iv_hi[0] ? lo + p.split_keys : job.iv_hi[0];
+                if (job.n_iv == 0 || hi < lo) hi = lo;
+                const int32_t rows = (slice < p.splits) ? (job.n_rows > kTile ? kTile : job.n_rows) : 0;
+                g.rows[st] = rows;
+                g.pos0[st] = (int32_t)job.q_pos0;
+                g.lo[st] = (int32_t)lo; g.hi[st] = (int32_t)hi;
+                int32_t end = g.hi[st];
+                if (p.causal && end > g.pos0[st] + rows) end = g.pos0[st] + rows;
+                g.cnt[st] = (rows > 0 && end > g.lo[st]) ? (end - g.lo[st] + kTile - 1) / kTile : 0;
+                g.n[st] = g.cnt[st];
+                g.n_max = g.cnt[st] > g.n_max ? g.cnt[st] : g.n_max;
+            }
         }
         sh->g = g;
     }
@@ -170,20 +194,41 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             mbar_arrive_expect_tx(bar_q, 2 * kTileBytes);
 #pragma unroll
             for (int st = 0; st < 2; ++st) {
-                const int row = sh->g.q_row0 + st * kTile;
+                const int row = sh->g.q_row0 + st * sh->g.q_st_stride;
                 tma_load_3d(sQ + st * kTileBytes, &tm_q, bar_q, 0, h, row);
                 tma_load_3d(sQ + st * kTileBytes + kHalfTileBytes, &tm_q, bar_q, 64, h, row);
             }
-            for (int i = 0; i < 2 * n_max; ++i) {              // items: K(0), V(0), K(1), V(1), ...
-                const int slot = i % kStages, fill = i / kStages;
-                if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p.status)) break;
-                const int jt = i >> 1, c0 = sh->g.cnt[0];
-                const int krow = sh->g.kv_row0 + (jt < c0 ? sh->g.lo[0] + jt * kTile : sh->g.lo[1] + (jt - c0) * kTile);
+            int filled = 0;                                    // ring items issued so far
+            auto load_tile = [&](const void *map, int krow) {
+                const int slot = filled % kStages, fill = filled / kStages;
+                if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p.status)) return false;
                 const uint32_t dst = sRing + slot * kTileBytes, bar = smem_u32(&sh->kv_full[slot]);
-                const void *map = (i & 1) ? (const void *)&tm_v : (const void *)&tm_k;
                 mbar_arrive_expect_tx(bar, kTileBytes);
                 tma_load_3d(dst, map, bar, 0, kvh, krow);
                 tma_load_3d(dst + kHalfTileBytes, map, bar, 64, kvh, krow);
+                ++filled;
+                return true;
+            };
+            bool ok = true;
+            if (!sh->g.dual) {
+                for (int i = 0; i < 2 * n_max && ok; ++i) {    // items: K(0), V(0), K(1), V(1), ...
+                    const int jt = i >> 1, c0 = sh->g.cnt[0];
+                    const int krow = sh->g.kv_row0 + (jt < c0 ? sh->g.lo[0] + jt * kTile : sh->g.lo[1] + (jt - c0) * kTile);
+                    ok = load_tile((i & 1) ? (const void *)&tm_v : (const void *)&tm_k, krow);
+                }
+            } else {
+                // Each stage has its own key slice; items in the order the MMA issuer consumes them:
+                // K_0(0), K_1(0), then per step V_0(j), K_0(j+1), V_1(j), K_1(j+1).
+                const int n0 = sh->g.n[0], n1 = sh->g.n[1];
+                const int base0 = sh->g.kv_row0 + sh->g.lo[0], base1 = sh->g.kv_row0 + sh->g.lo[1];
+                if (n0 > 0) ok = load_tile(&tm_k, base0);
+                if (ok && n1 > 0) ok = load_tile(&tm_k, base1);
+                for (int j = 0; j < n_max && ok; ++j) {
+                    if (ok && j < n0) ok = load_tile(&tm_v, base0 + j * kTile);
+                    if (ok && j + 1 < n0) ok = load_tile(&tm_k, base0 + (j + 1) * kTile);
+                    if (ok && j < n1) ok = load_tile(&tm_v, base1 + j * kTile);
+                    if (ok && j + 1 < n1) ok = load_tile(&tm_k, base1 + (j + 1) * kTile);
+                }
             }
         }
         __syncwarp();
@@ -219,30 +264,64 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             };
 
             const int n_st[2] = {sh->g.n[0], sh->g.n[1]};
-            bool ok = wait_bar(smem_u32(&sh->bar_q), 0, sh, p.status) && kv_wait(0);
-            if (ok) {
-                if (n_st[0] > 0) issue_qk(0, 0);
-                if (n_st[1] > 0) issue_qk(1, 0);
-                kv_release(0);
-            }
-            for (int j = 0; j < n_max && ok; ++j) {
-                const bool has_next = j + 1 < n_max;
-                ok = kv_wait(2 * j + 1);                       // V(j)
+            bool ok = wait_bar(smem_u32(&sh->bar_q), 0, sh, p.status);
+            if (ok && !sh->g.dual) {
+                ok = kv_wait(0);
+                if (ok) {
+                    if (n_st[0] > 0) issue_qk(0, 0);
+                    if (n_st[1] > 0) issue_qk(1, 0);
+                    kv_release(0);
+                }
+                for (int j = 0; j < n_max && ok; ++j) {
+                    const bool has_next = j + 1 < n_max;
+                    ok = kv_wait(2 * j + 1);                   // V(j)
+#pragma unroll
+                    for (int st = 0; st < 2 && ok; ++st) {
+                        if (j < n_st[st]) {
+                            ok = wait_bar(smem_u32(&sh->p_ready[st]), j & 1, sh, p.status);
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_pv(st, 2 * j + 1, j > 0);
+                            if (j == n_st[st] - 1) tc_commit(smem_u32(&sh->o_final[st]));
+                        }
+                        if (st == 0 && has_next) { ok = kv_wait(2 * j + 2); if (!ok) break; }   // K(j+1)
+                        if (j + 1 < n_st[st]) issue_qk(st, 2 * j + 2);
+                    }
+                    if (!ok) break;
+                    kv_release(2 * j + 1);
+                    if (has_next) kv_release(2 * j + 2);
+                }
+            } else if (ok) {
+                // Dual: every ring item has one consumer; items arrive in the order used here.
+                int item = 0;
 #pragma unroll
                 for (int st = 0; st < 2 && ok; ++st) {
-                    if (j < n_st[st]) {
-                        ok = wait_bar(smem_u32(&sh->p_ready[st]), j & 1, sh, p.status);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_pv(st, 2 * j + 1, j > 0);
-                        if (j == n_st[st] - 1) tc_commit(smem_u32(&sh->o_final[st]));
+                    if (n_st[st] > 0) {
+                        ok = kv_wait(item);
+                        if (ok) { issue_qk(st, item); kv_release(item); ++item; }
                     }
-                    if (st == 0 && has_next) { ok = kv_wait(2 * j + 2); if (!ok) break; }   // K(j+1)
-                    if (j + 1 < n_st[st]) issue_qk(st, 2 * j + 2);
                 }
-                if (!ok) break;
-                kv_release(2 * j + 1);
-                if (has_next) kv_release(2 * j + 2);
+                for (int j = 0; j < n_max && ok; ++j) {
+#pragma unroll
+                    for (int st = 0; st < 2 && ok; ++st) {
+                        if (j < n_st[st]) {
+                            ok = wait_bar(smem_u32(&sh->p_ready[st]), j & 1, sh, p.status) && kv_wait(item);   // P_st(j), V_st(j)
+                            if (!ok) break;
+                            tc_fence_after();
+                            issue_pv(st, item, j > 0);
+                            if (j == n_st[st] - 1) tc_commit(smem_u32(&sh->o_final[st]));
+                            kv_release(item);
+                            ++item;
+                        }
+                        if (j + 1 < n_st[st]) {
+                            ok = kv_wait(item);                // K_st(j+1)
+                            if (!ok) break;
+                            issue_qk(st, item);
+                            kv_release(item);
+                            ++item;
+                        }
+                    }
+                }
             }
         }
         __syncwarp();
@@ -260,15 +339,17 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const uint32_t bar_s = smem_u32(&sh->s_full[st]), bar_p = smem_u32(&sh->p_ready[st]);
         // Per interval: where it ends, and the first key position that some row of this stage cannot
         // see (tiles reaching past it need the mask).
-        const int pos0 = sh->g.pos0[st], my_pos = pos0 + row_in_tile, cnt0 = sh->g.cnt[0];
+        // (Dual launches: interval st is this stage's own key slice and the walk never changes interval.)
+        const bool dual = sh->g.dual != 0;
+        const int pos0 = sh->g.pos0[st], my_pos = pos0 + row_in_tile, cnt0 = dual ? 0x7fffffff : sh->g.cnt[0];
         int iv_full[2], iv_mine[2];
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
-            const int hi_t = sh->g.hi[t];
+            const int hi_t = dual ? sh->g.hi[st] : sh->g.hi[t];
             iv_full[t] = (p.causal && pos0 + 1 < hi_t) ? pos0 + 1 : hi_t;
             iv_mine[t] = (p.causal && my_pos + 1 < hi_t) ? my_pos + 1 : hi_t;
         }
-        int k0 = sh->g.lo[0], cur = 0;
+        int k0 = dual ? sh->g.lo[st] : sh->g.lo[0], cur = 0;
 
         float m_ref = -INFINITY, l_run = 0.f;                // m_ref in log2 units of the scaled scores
         bool ok = true;
@@ -358,7 +439,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const bool valid = row_in_tile < sh->g.rows[st];
             const bool empty = (l_run == 0.f);
             const float inv = empty ? 0.f : 1.f / l_run;
-            const int64_t row = (int64_t)sh->g.out_row0 + st * kTile + row_in_tile;
+            const int64_t row = (int64_t)sh->g.out_row0 + st * sh->g.out_st_stride + row_in_tile;
             const int64_t obase = (row * p.Hq + h) * kHeadDim;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -468,7 +549,9 @@ int launch_attn_bf16(const AttnParams &p, cudaStream_t stream)
     if (p.cu_seqlens) tiles += p.B;
     if (tiles > 0x7fffffff || p.Hq > 65535) { set_error("pec_prefill_attn: grid too large"); return PEC_ERR_UNSUPPORTED; }
     if (p.splits < 1 || p.splits > 65535) { set_error("pec_prefill_attn: bad split count"); return PEC_ERR_INVALID_ARG; }
-    dim3 grid((unsigned)tiles, (unsigned)p.Hq, (unsigned)p.splits);
+    if (p.splits > 1 && p.total_rows > kTile) { set_error("pec_prefill_attn: split launches take at most 128 query rows"); return PEC_ERR_UNSUPPORTED; }
+    // Split launches are dual: each CTA's two stages take two consecutive key slices.
+    dim3 grid((unsigned)tiles, (unsigned)p.Hq, (unsigned)(p.splits > 1 ? (p.splits + 1) / 2 : 1));
     attn_bf16_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, p);
     const cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("pec_prefill_attn: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }

@@ -5,8 +5,10 @@
 // HBM-bound: the keys and values of the range are read once (2 * keys * Hkv * 128 * 2 bytes).  The
 // g = Hq / Hkv query heads that share a KV head are laid out as the g rows of one 128-row tile of
 // that KV head, so the tensor-core prefill kernel does the work with every K/V byte used by all g
-// heads; the key range is cut into slices, one CTA per (KV head, slice), whose partial (O, LSE)
-// go to scratch memory and are combined by the small kernel below (same LSE merge as pec_attn_merge).
+// heads; the key range is cut into slices, one CTA per (KV head, pair of slices) - its two stages
+// take one slice each so that one slice's softmax overlaps the other's MMAs - whose partial
+// (O, LSE) go to scratch memory and are combined by the small kernel below (same LSE merge as
+// pec_attn_merge).
 #include <cuda_bf16.h>
 #include <cmath>
 #include <mutex>
