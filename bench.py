@@ -353,6 +353,43 @@ def run_decode(args):
                       "max_abs_err_vs_oracle": err}), flush=True)
 
 
+def run_linear(args):
+    """Extra line: the QKV-generation GEMM of a Llama-3-8B-shaped layer (Eq. 2) on 32768 tokens."""
+    from paper_2409_15104_b200 import binding
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    M, K, N = 32768, 4096, (32 + 2 * 8) * 128
+    seed = workloads.BASE_SEED + 7
+    x = workloads.normal_tensor(seed, 1, (M, K), torch.bfloat16).to(dev)
+    w = (workloads.normal_tensor(seed, 2, (N, K), torch.float32) / K ** 0.5).to(torch.bfloat16).to(dev)
+    y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    for _ in range(max(args.warmup, 3)):
+        binding.pec_linear(x, w, y=y)
+    torch.cuda.synchronize()
+    steps = min(args.steps, 50)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        binding.pec_linear(x, w, y=y)
+    e1.record()
+    torch.cuda.synchronize()
+    binding.check_status()
+    ms = e0.elapsed_time(e1) / steps
+    tf = 2.0 * M * N * K / (ms * 1e-3) / 1e12
+    peaks = load_peaks()
+    import oracle
+    rows = [0, 1, 127, 128, 4095, M - 1]
+    want = oracle.linear(x[rows].cpu(), w.cpu())
+    err = float(np.abs(y[rows].float().cpu().double().numpy() - want).max())
+    print(json.dumps({"metric": "QKV-generation GEMM TFLOP/s (extra line, not the headline)", "value": tf, "unit": "TFLOP/s",
+                      "ms_per_step": ms, "steps": steps, "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": f"linear: x [{M},{K}] times w [{N},{K}]^T", "l2": "operands and output (752 MB) exceed L2"},
+                      "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+                                   "frac": tf / peaks["bf16_sustained"], "traffic": None,
+                                   "peak_source": peaks["source"] + " sustained cuBLAS bf16"},
+                      "max_abs_err_vs_oracle_sampled_rows": err}), flush=True)
+
+
 def _short_batch(wl, dev, seed_offset=0):
     lens = workloads.short_lengths(wl.seed, wl.short_batch)
     cu = workloads.cu_seqlens(lens)
@@ -458,7 +495,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode"], default="c3")
+    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode", "linear"], default="c3")
     ap.add_argument("--reference-seconds", type=float, default=0.0,
                     help="--impl reference: CPU seconds per step (default: 90 s spread over the steps, 0.15-20 s each)")
     ap.add_argument("--profile", action="store_true",
@@ -467,6 +504,9 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.workload == "decode":
         run_decode(args)
+        return
+    if args.workload == "linear":
+        run_linear(args)
         return
     wl = workloads.WORKLOADS[args.workload]
     if args.workload == "c2":

@@ -281,6 +281,19 @@ typedef struct {
 } pec_sp_choice;
 int pec_select_sp(const pec_sp_inputs *in, pec_sp_choice *out);
 
+/*
+ * y = x w^T, bf16 inputs and output, fp32 accumulation: the dense steps on either side of the
+ * attention.  With w = the W_Q, W_K, W_V of all heads stacked row-wise it is the QKV generation
+ * of Eq. 2 (y is then the fused [T, (Hq + 2 Hkv) * D] tensor whose column slices are the q, k, v
+ * of pec_prefill_attn, addressed through its stride arguments); with w = W_L^T it is the
+ * post-self-attention linear layer of Eq. 5.
+ * x: device [M, K], w: device [N, K], y: device [M, N]; row-major with row strides in elements
+ * (multiples of 8), 16-byte aligned; N and K multiples of 8.  `status`: required device word, used as
+ * in pec_attn_args.  Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.
+ */
+int pec_linear(const void *x, int64_t x_stride, const void *w, int64_t w_stride, void *y, int64_t y_stride,
+               int64_t M, int32_t N, int32_t K, int32_t *status, void *cuda_stream);
+
 /* Text describing the last non-zero return on this thread (never NULL). */
 const char *pec_last_error(void);
 

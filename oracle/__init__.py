@@ -11,6 +11,7 @@ from .reference import (  # noqa: F401
     merge_n,
     sp_volumes,
     select_sp,
+    linear,
     plan_partitions,
     partition_intervals,
     oracle_threads,

@@ -277,3 +277,10 @@ def select_sp(s, d, n_h, n_kv, d_h, T, G, elem_bytes, node_bw, gpu_flops):
     order = [("megatron", "megatron"), ("megatron", "ulysses"), ("ulysses", "megatron"), ("ulysses", "ulysses")]
     best = min(order, key=lambda c: (times[c], order.index(c)))
     return best, times
+
+
+# --------------------------------------------------------------------------- dense steps (Eq. 2, Eq. 5)
+def linear(x, w):
+    """y = x w^T in fp64 (numpy matmul): QKV generation (Eq. 2) with the per-head weights stacked
+    row-wise in w, or the post-self-attention linear layer (Eq. 5) with w = W_L^T."""
+    return _as_f32(x).astype(np.float64) @ _as_f32(w).astype(np.float64).T

@@ -87,7 +87,7 @@ class pec_plan(ctypes.Structure):
 
 
 EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_attn_merge_n", "pec_plan_partitions",
-           "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size", "pec_decode_attn_static", "pec_select_sp")
+           "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size", "pec_decode_attn_static", "pec_select_sp", "pec_linear")
 PEC_DECODE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 PEC_MERGE_MAX_PARTS = 16
 
@@ -121,6 +121,10 @@ def load():
     lib.pec_decode_attn_static.argtypes = [ctypes.POINTER(pec_decode_args), ctypes.c_void_p]
     lib.pec_decode_workspace_size.restype = ctypes.c_size_t
     lib.pec_decode_workspace_size.argtypes = [ctypes.POINTER(pec_decode_args)]
+    lib.pec_linear.restype = ctypes.c_int
+    lib.pec_linear.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+                               ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                               ctypes.c_void_p]
     lib.pec_select_sp.restype = ctypes.c_int
     lib.pec_select_sp.argtypes = [ctypes.POINTER(pec_sp_inputs), ctypes.POINTER(pec_sp_choice)]
     lib.pec_last_error.restype = ctypes.c_char_p
@@ -308,6 +312,21 @@ def pec_decode_attn(q, k, v, *, kv_lo=0, kv_hi=None, num_splits=0, softmax_scale
     a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel()
     _check(lib.pec_decode_attn(ctypes.byref(a), _stream_ptr(stream)))
     return o, lse
+
+
+def pec_linear(x, w, y=None, stream=None):
+    """y = x w^T (bf16, fp32 accumulation); x [M,K], w [N,K] CUDA tensors with contiguous rows; returns y [M,N]."""
+    lib = load()
+    assert x.is_cuda and w.is_cuda and x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
+    assert x.stride(1) == 1 and w.stride(1) == 1 and x.shape[1] == w.shape[1]
+    M, K = x.shape
+    N = w.shape[0]
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    assert y.stride(1) == 1
+    _check(lib.pec_linear(x.data_ptr(), x.stride(0), w.data_ptr(), w.stride(0), y.data_ptr(), y.stride(0), M, N, K,
+                          status_word(x.device).data_ptr(), _stream_ptr(stream)))
+    return y
 
 
 def pec_select_sp(s, d, n_h, n_kv, d_h, T, G, elem_bytes=2.0, node_bw=1.0, gpu_flops=1.0):

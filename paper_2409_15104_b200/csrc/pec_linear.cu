@@ -1,0 +1,221 @@
+// y = x w^T in bf16 with fp32 accumulation: the dense steps either side of the attention - QKV
+// generation (Eq. 2, with W_Q, W_K, W_V of all heads stacked row-wise in w so that y is the fused
+// [T, (Hq + 2 Hkv) * 128] tensor whose slices pec_prefill_attn reads through strides) and the
+// post-self-attention linear layer (Eq. 5).
+//
+// One CTA = one 128 x 256 tile of y.  Warp 5 streams 128 x 64 tiles of x and 256 x 64 tiles of w
+// by TMA into a 4-slot ring (128-byte swizzle, both operands K-major); warp 4 issues tcgen05.mma
+// 128 x 256 x 16 (4 per ring slot) into a 256-column fp32 accumulator in tensor memory; warps 0-3
+// read the accumulator back (one output row per thread), round to bf16 and store.  Tensor-bound:
+// 2 * M * N * K operations; per ring slot the MMAs read 48 KB of shared memory in 512 cycles.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include "pec_internal.h"
+#include "pec_sm100.cuh"
+
+namespace pec {
+using namespace sm100;
+
+namespace lin {
+constexpr int kBM = 128, kBN = 256, kBK = 64;
+constexpr int kSlots = 4;
+constexpr int kThreads = 192;                               // 4 epilogue warps, MMA warp, loader warp
+constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2, kSlotBytes = kABytes + kBBytes;
+constexpr uint32_t kTmemCols = 256;
+constexpr long long kWaitCycles = 2000000000LL;
+
+struct Shared {
+    uint64_t full[kSlots], empty[kSlots], acc_full;
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+constexpr size_t kSmemBytes = kSlots * kSlotBytes + 1024 + sizeof(Shared);
+
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *sh, int32_t *status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait_suspend(bar, parity, 2000)) {
+        if (sh->abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            sh->abort_flag = 1;
+            if (status) atomicExch(status, (int)PEC_ERR_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void *tmap, uint32_t bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+              __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t *status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t ring = (raw + 1023u) & ~1023u;
+    Shared *sh = reinterpret_cast<Shared *>(smem_raw + (ring - raw) + kSlots * kSlotBytes);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t m0 = (int64_t)blockIdx.x * kBM;            // x tiles fastest: neighbours share the w tile in L2
+    const int n0 = blockIdx.y * kBN;
+    const int n_kb = (K + kBK - 1) / kBK;
+
+    if (tid == 0) {
+        sh->abort_flag = (status && *reinterpret_cast<volatile int32_t *>(status) != 0) ? 1 : 0;
+        for (int s = 0; s < kSlots; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
+        mbar_init(smem_u32(&sh->acc_full), 1);
+        mbar_init_fence();
+        prefetch_tmap(&tm_x); prefetch_tmap(&tm_w);
+    }
+    __syncthreads();
+    if (sh->abort_flag) return;                               // an earlier launch's wait expired (uniform)
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&sh->tmem_base), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh->tmem_base;
+
+    if (warp == 5) {
+        if (lane == 0) {
+            for (int kb = 0; kb < n_kb; ++kb) {
+                const int slot = kb % kSlots, fill = kb / kSlots;
+                if (fill > 0 && !wait_bar(smem_u32(&sh->empty[slot]), (fill - 1) & 1, sh, status)) break;
+                const uint32_t a = ring + slot * kSlotBytes, bar = smem_u32(&sh->full[slot]);
+                mbar_arrive_expect_tx(bar, kSlotBytes);
+                tma_load_2d(a, &tm_x, bar, kb * kBK, (int)m0);
+                tma_load_2d(a + kABytes, &tm_w, bar, kb * kBK, n0);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 4) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(kBM, kBN, 0, 0);
+            bool ok = true;
+            for (int kb = 0; kb < n_kb && ok; ++kb) {
+                const int slot = kb % kSlots;
+                ok = wait_bar(smem_u32(&sh->full[slot]), (kb / kSlots) & 1, sh, status);
+                if (!ok) break;
+                const uint32_t a = ring + slot * kSlotBytes, b = a + kABytes;
+#pragma unroll
+                for (int ks = 0; ks < kBK / 16; ++ks)
+                    mma_ss(tmem, smem_desc_sw128(a + ks * 32u, 16, 1024), smem_desc_sw128(b + ks * 32u, 16, 1024), idesc,
+                           (kb > 0 || ks > 0) ? 1u : 0u);
+                tc_commit(smem_u32(&sh->empty[slot]));
+            }
+            if (ok) tc_commit(smem_u32(&sh->acc_full));
+        }
+        __syncwarp();
+    } else {
+        // epilogue: thread = output row (TMEM lane); 256 accumulator columns in chunks of 32
+        const bool ok = __all_sync(0xffffffffu, n_kb == 0 || wait_bar(smem_u32(&sh->acc_full), 0, sh, status));
+        if (ok) {
+            tc_fence_after();
+            const int64_t row = m0 + warp * 32 + lane;
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < kBN / 32; ++c) {
+                uint32_t r[32];
+                if (n_kb == 0) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;
+                } else {
+                    tmem_ld32(taddr + c * 32, r);             // warp-wide; only the stores are predicated
+                }
+                if (row < M) {
+                    __nv_bfloat16 *dst = y + row * y_stride + n0 + c * 32;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        if (n0 + c * 32 + i < N) {            // N is a multiple of 8
+                            uint4 pk;
+                            pk.x = pack_bf16(__uint_as_float(r[i + 0]), __uint_as_float(r[i + 1]));
+                            pk.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                            pk.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+                            pk.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+                            *reinterpret_cast<uint4 *>(dst + i) = pk;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// [rows, cols] bf16 matrix, row stride in elements; box = 64 columns x box_rows rows.
+static bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t stride, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)stride * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+}  // namespace lin
+}  // namespace pec
+
+using namespace pec;
+
+extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_t w_stride, void *y, int64_t y_stride,
+                          int64_t M, int32_t N, int32_t K, int32_t *status, void *cuda_stream)
+{
+    if (!x || !w || !y || !status) { set_error("pec_linear: x, w, y and status must be non-NULL"); return PEC_ERR_INVALID_ARG; }
+    if (M < 0 || N < 1 || K < 1 || M >= ((int64_t)1 << 31)) { set_error("pec_linear: need 0 <= M < 2^31, N >= 1, K >= 1"); return PEC_ERR_INVALID_ARG; }
+    if (N % 8 != 0 || K % 8 != 0) { set_error("pec_linear: N and K must be multiples of 8"); return PEC_ERR_UNSUPPORTED; }
+    if (x_stride < K || w_stride < K || y_stride < N) { set_error("pec_linear: a row stride is smaller than the row"); return PEC_ERR_INVALID_ARG; }
+    if (x_stride % 8 != 0 || w_stride % 8 != 0 || y_stride % 8 != 0 || (reinterpret_cast<uintptr_t>(x) & 15u) ||
+        (reinterpret_cast<uintptr_t>(w) & 15u) || (reinterpret_cast<uintptr_t>(y) & 15u) || (reinterpret_cast<uintptr_t>(status) & 3u)) {
+        set_error("pec_linear: x, w, y must be 16-byte aligned with row strides that are multiples of 8 elements");
+        return PEC_ERR_ALIGNMENT;
+    }
+    if (M == 0) return PEC_OK;
+    CUtensorMap tm_x, tm_w;
+    if (!lin::make_map(&tm_x, x, M, K, x_stride, lin::kBM) || !lin::make_map(&tm_w, w, N, K, w_stride, lin::kBN)) {
+        set_error("pec_linear: cuTensorMapEncodeTiled failed");
+        return PEC_ERR_CUDA;
+    }
+    if (cudaFuncSetAttribute(lin::linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::kSmemBytes) != cudaSuccess) {
+        set_error("pec_linear: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
+        return PEC_ERR_CUDA;
+    }
+    const int64_t gm = (M + lin::kBM - 1) / lin::kBM, gn = (N + lin::kBN - 1) / lin::kBN;
+    if (gn > 65535) { set_error("pec_linear: N too large"); return PEC_ERR_UNSUPPORTED; }
+    dim3 grid((unsigned)gm, (unsigned)gn);
+    lin::linear_kernel<<<grid, lin::kThreads, lin::kSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(
+        tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, status);
+    const cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) { set_error("pec_linear: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
+    return PEC_OK;
+}

@@ -284,3 +284,36 @@ def test_non_causal_partition_of_a_chunk(pec, dtype):
                                       num_parts=P, part_align=32, causal=False)
         pec.check_status()
         compare(o, lse, *want, *TOL[dtype], f"non-causal chunk x partition {p}")
+
+
+# ------------------------------------------------------------------ dense steps either side of the attention
+@pytest.mark.parametrize("M,N,K", [(1, 8, 8), (128, 256, 64), (130, 264, 72), (1000, 768, 512), (257, 6144, 4096),
+                                   (4096, 128, 1024)])
+def test_linear_matches_oracle(pec, M, N, K):
+    x = workloads.normal_tensor(15000 + M, 1, (M, K), torch.bfloat16)
+    w = (workloads.normal_tensor(15001 + N, 2, (N, K), torch.float32) / K ** 0.5).to(torch.bfloat16)
+    want = oracle.linear(x, w)
+    y = pec.pec_linear(x.to(DEV), w.to(DEV))
+    pec.check_status()
+    err = np.abs(y.float().cpu().double().numpy() - want).max()
+    print(f"[parity] linear {M}x{N}x{K}: max|dy| = {err:.3e}")
+    assert err <= 2e-2                                   # outputs ~ N(0,1); bf16 rounding of the result dominates
+
+
+def test_attention_layer_steps_chain_through_strides(pec):
+    """Eq. 2 -> Eq. 3 -> Eq. 5 on the GPU: fused QKV projection, attention reading q/k/v as strided slices of
+    it, output projection; each step checked against the oracle applied to that step's actual inputs."""
+    T, d, hq, hkv = 600, 512, 4, 2
+    e = workloads.normal_tensor(16000, 1, (T, d), torch.bfloat16)
+    w_qkv = (workloads.normal_tensor(16001, 2, ((hq + 2 * hkv) * 128, d), torch.float32) / d ** 0.5).to(torch.bfloat16)
+    w_l = (workloads.normal_tensor(16002, 3, (d, hq * 128), torch.float32) / (hq * 128) ** 0.5).to(torch.bfloat16)
+    qkv = pec.pec_linear(e.to(DEV), w_qkv.to(DEV))
+    fused = qkv.view(T, hq + 2 * hkv, 128)
+    q, k, v = fused[:, :hq], fused[:, hq:hq + hkv], fused[:, hq + hkv:]
+    o, lse = pec.pec_prefill_attn(q, k, v)
+    out = pec.pec_linear(o.view(T, hq * 128), w_l.to(DEV))
+    pec.check_status()
+    assert np.abs(qkv.float().cpu().double().numpy() - oracle.linear(e, w_qkv)).max() <= 2e-2
+    want = oracle.prefill_attn(q.cpu(), k.cpu(), v.cpu(), seq_len=T)
+    compare(o, lse, *want, 2e-2, 1e-3, "attention on projected q, k, v")
+    assert np.abs(out.float().cpu().double().numpy() - oracle.linear(o.view(T, hq * 128).cpu(), w_l)).max() <= 2e-2

@@ -154,3 +154,18 @@ def test_decode_validates_on_the_host_and_sizes_its_workspace():
         assert lib.pec_decode_attn(ctypes.byref(a), None) == code, field
         assert lib.pec_decode_workspace_size(ctypes.byref(a)) == 0
         setattr(a, field, old)
+
+
+def test_linear_validates_on_the_host():
+    f = binding.load().pec_linear
+    ok = dict(x=4096, xs=64, w=8192, ws=64, y=12288, ys=32, M=10, N=32, K=64, st=16384)
+
+    def call(**over):
+        a = {**ok, **over}
+        return f(a["x"], a["xs"], a["w"], a["ws"], a["y"], a["ys"], a["M"], a["N"], a["K"], a["st"], None)
+
+    assert call(M=0) == 0
+    assert call(x=None) == -1 and call(st=None) == -1 and call(M=-1) == -1 and call(N=0) == -1
+    assert call(N=30) == -2 and call(K=60, xs=64) == -2
+    assert call(xs=32) == -1 and call(ys=16) == -1
+    assert call(x=4100) == -3 and call(ws=68) == -3

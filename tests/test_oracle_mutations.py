@@ -115,6 +115,7 @@ PY_MUTATIONS = {
     "kv prefix ignored": ("        hi = min(hi, kv_len)\n", ""),
     "Megatron attention term not divided by T": ("qkv / T + 4 * (s * T) ** 2 * d / T + out_proj", "qkv / T + 4 * (s * T) ** 2 * d + out_proj"),
     "Ulysses all-to-all counts G not G-1": ("a2a = 2 * s * (n_h + n_kv) * d_h * (G - 1)", "a2a = 2 * s * (n_h + n_kv) * d_h * G"),
+    "linear without the transpose of w": ('@ _as_f32(w).astype(np.float64).T', '@ _as_f32(w).astype(np.float64)[:, ::-1].T'),
     "MLP parameter volume 4 d^2": ("(8 * d * d * (T - 1) * G / T, 16 * s * d * d)", "(4 * d * d * (T - 1) * G / T, 16 * s * d * d)"),
 }
 
@@ -129,6 +130,6 @@ def test_a_mistake_in_the_python_oracle_is_caught(name, monkeypatch):
     mod.__file__ = ref.__file__
     exec(compile(src.replace(old, new), "reference_mutant.py", "exec"), mod.__dict__)
     for attr in ("attn_rows", "prefill_attn", "varlen_attn", "merge", "merge_n", "plan_partitions",
-                 "partition_intervals", "sp_volumes", "select_sp"):
+                 "partition_intervals", "sp_volumes", "select_sp", "linear"):
         monkeypatch.setattr(oracle, attr, getattr(mod, attr))
     assert _some_pin_fails(_all_oracle_pins()), f"no pin noticed: {name}"

@@ -333,3 +333,19 @@ def test_bf16_inputs_widen_exactly():
     a = oracle.attn_rows(q, np.arange(S), k, v, [(0, S)], True)
     b = oracle.attn_rows(q.float().numpy(), np.arange(S), k.float().numpy(), v.float().numpy(), [(0, S)], True)
     np.testing.assert_array_equal(a[0], b[0])
+
+
+# ------------------------------------------------------------------ dense steps
+def test_linear_matches_loops_identity_and_per_head_stacking():
+    """Eq. 2 / Eq. 5 as y = x w^T: explicit loops on a tiny case, identity weights, and stacking the
+    per-head W_Q, W_K, W_V row-wise gives the per-head products side by side."""
+    x, w = _rand((5, 6), 201), _rand((4, 6), 202)
+    y = oracle.linear(x, w)
+    for i in range(5):
+        for j in range(4):
+            assert abs(y[i, j] - sum(float(x[i, c]) * float(w[j, c]) for c in range(6))) < 1e-12
+    np.testing.assert_array_equal(oracle.linear(x, np.eye(6, dtype=np.float32)), x.astype(np.float64))
+    wq, wk = _rand((3, 6), 203), _rand((2, 6), 204)
+    both = oracle.linear(x, np.concatenate([wq, wk]))
+    np.testing.assert_array_equal(both[:, :3], oracle.linear(x, wq))
+    np.testing.assert_array_equal(both[:, 3:], oracle.linear(x, wk))
