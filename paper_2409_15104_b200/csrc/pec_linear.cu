@@ -3,13 +3,15 @@
 // [T, (Hq + 2 Hkv) * 128] tensor whose slices pec_prefill_attn reads through strides) and the
 // post-self-attention linear layer (Eq. 5).
 //
-// One CTA = one 128 x 256 tile of y.  Warp 5 streams 128 x 64 tiles of x and 256 x 64 tiles of w
-// by TMA into a 2-slot ring (128-byte swizzle, both operands K-major); warp 4 issues tcgen05.mma
-// 128 x 256 x 16 (4 per ring slot) into a 256-column fp32 accumulator in tensor memory; warps 0-3
-// read the accumulator back (one output row per thread), round to bf16 and store.  Two CTAs fit on
-// an SM (2 x 96 KB of shared memory, 2 x 256 TMEM columns), so one CTA's epilogue and load latency
-// hide under the other's MMAs (measured 8 % faster than one CTA with a 4-slot ring).  Tensor-bound:
-// 2 * M * N * K operations; per ring slot the MMAs read 48 KB of shared memory in 512 cycles.
+// A cluster of two CTAs computes one 256 x 256 tile of y with 256-row MMAs (cta_group::2).  Per K
+// step of 64 each CTA loads, by TMA into a 3-slot ring (128-byte swizzle, both operands K-major),
+// its own 128 rows of x and 128 of the 256 rows of w - half the shared-memory operand traffic per
+// operation of a single-CTA 128 x 256 tile - and keeps its 128 rows of the fp32 accumulator in its
+// own tensor memory (256 columns).  The even-ranked CTA (the leader) issues every tcgen05.mma; both
+// CTAs' loads count on the leader's "full" barrier and the leader's commits arrive on both CTAs'
+// barriers.  Warps 0-3 of each CTA read its accumulator rows back, round to bf16 and store.  Two
+// CTAs (of different pairs) fit on an SM (2 x 96 KB, 2 x 256 TMEM columns), so one's epilogue and
+// load latency hide under the other's MMAs.  Tensor-bound: 2 * M * N * K operations.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -21,9 +23,11 @@ using namespace sm100;
 
 namespace lin {
 constexpr int kBM = 128, kBN = 256, kBK = 64;
-constexpr int kSlots = 2;                                   // 96 KB per CTA: two CTAs share an SM
+constexpr int kSlots = 3;                                   // 96 KB per CTA: two CTAs share an SM
 constexpr int kThreads = 192;                               // 4 epilogue warps, MMA warp, loader warp
-constexpr uint32_t kABytes = kBM * kBK * 2, kBBytes = kBN * kBK * 2, kSlotBytes = kABytes + kBBytes;
+constexpr uint32_t kABytes = kBM * kBK * 2;                 // this CTA's 128 rows of x
+constexpr uint32_t kWBytes = 128 * kBK * 2;                 // this CTA's half of the 256 rows of w
+constexpr uint32_t kSlotBytes = kABytes + kWBytes;          // 32 KB
 constexpr uint32_t kTmemCols = 256;
 constexpr long long kWaitCycles = 2000000000LL;
 
@@ -49,23 +53,17 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *
     return true;
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void *tmap, uint32_t bar, int c0, int c1)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1) : "memory");
-}
-
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 2)
 linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-              __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t *status)
+                   __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t *status)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;
     Shared *sh = reinterpret_cast<Shared *>(smem_raw + (ring - raw) + kSlots * kSlotBytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int64_t m0 = (int64_t)blockIdx.x * kBM;            // x tiles fastest: neighbours share the w tile in L2
+    const uint32_t rank = cluster_ctarank();                  // 0 = leader
+    const int64_t m0 = (int64_t)(blockIdx.x >> 1) * (2 * kBM) + rank * kBM;
     const int n0 = blockIdx.y * kBN;
     const int n_kb = (K + kBK - 1) / kBK;
 
@@ -77,10 +75,12 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
         prefetch_tmap(&tm_x); prefetch_tmap(&tm_w);
     }
     __syncthreads();
-    if (sh->abort_flag) return;                               // an earlier launch's wait expired (uniform)
+    // No early exit here: the two CTAs of a pair must take every collective step together (a CTA that
+    // starts with the abort flag set simply lets its waits fail at once).
+    cluster_sync();                                           // both CTAs' barriers exist before anyone signals them
     if (warp == 0) {
-        tmem_alloc(smem_u32(&sh->tmem_base), kTmemCols);
-        tmem_relinquish();
+        tmem_alloc_pair(smem_u32(&sh->tmem_base), kTmemCols);
+        tmem_relinquish_pair();
     }
     tc_fence_before();
     __syncthreads();
@@ -92,16 +92,17 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
             for (int kb = 0; kb < n_kb; ++kb) {
                 const int slot = kb % kSlots, fill = kb / kSlots;
                 if (fill > 0 && !wait_bar(smem_u32(&sh->empty[slot]), (fill - 1) & 1, sh, status)) break;
-                const uint32_t a = ring + slot * kSlotBytes, bar = smem_u32(&sh->full[slot]);
-                mbar_arrive_expect_tx(bar, kSlotBytes);
-                tma_load_2d(a, &tm_x, bar, kb * kBK, (int)m0);
-                tma_load_2d(a + kABytes, &tm_w, bar, kb * kBK, n0);
+                const uint32_t a = ring + slot * kSlotBytes;
+                const uint32_t bar = leader_addr(smem_u32(&sh->full[slot]));
+                if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[slot]), 2 * kSlotBytes);   // both CTAs' bytes
+                tma_load_2d_pair(a, &tm_x, bar, kb * kBK, (int)m0);
+                tma_load_2d_pair(a + kABytes, &tm_w, bar, kb * kBK, n0 + (int)rank * 128);
             }
         }
         __syncwarp();
     } else if (warp == 4) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16_f32(kBM, kBN, 0, 0);
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(2 * kBM, kBN, 0, 0);
             bool ok = true;
             for (int kb = 0; kb < n_kb && ok; ++kb) {
                 const int slot = kb % kSlots;
@@ -110,15 +111,14 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
                 const uint32_t a = ring + slot * kSlotBytes, b = a + kABytes;
 #pragma unroll
                 for (int ks = 0; ks < kBK / 16; ++ks)
-                    mma_ss(tmem, smem_desc_sw128(a + ks * 32u, 16, 1024), smem_desc_sw128(b + ks * 32u, 16, 1024), idesc,
-                           (kb > 0 || ks > 0) ? 1u : 0u);
-                tc_commit(smem_u32(&sh->empty[slot]));
+                    mma_ss_pair(tmem, smem_desc_sw128(a + ks * 32u, 16, 1024), smem_desc_sw128(b + ks * 32u, 16, 1024), idesc,
+                                (kb > 0 || ks > 0) ? 1u : 0u);
+                tc_commit_pair(smem_u32(&sh->empty[slot]));
             }
-            if (ok) tc_commit(smem_u32(&sh->acc_full));
+            if (ok) tc_commit_pair(smem_u32(&sh->acc_full));
         }
         __syncwarp();
     } else {
-        // epilogue: thread = output row (TMEM lane); 256 accumulator columns in chunks of 32
         const bool ok = __all_sync(0xffffffffu, n_kb == 0 || wait_bar(smem_u32(&sh->acc_full), 0, sh, status));
         if (ok) {
             tc_fence_after();
@@ -127,17 +127,12 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
 #pragma unroll 1
             for (int c = 0; c < kBN / 32; ++c) {
                 uint32_t r[32];
-                if (n_kb == 0) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = 0u;
-                } else {
-                    tmem_ld32(taddr + c * 32, r);             // warp-wide; only the stores are predicated
-                }
+                tmem_ld32(taddr + c * 32, r);                 // warp-wide; only the stores are predicated
                 if (row < M) {
                     __nv_bfloat16 *dst = y + row * y_stride + n0 + c * 32;
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
-                        if (n0 + c * 32 + i < N) {            // N is a multiple of 8
+                        if (n0 + c * 32 + i < N) {
                             uint4 pk;
                             pk.x = pack_bf16(__uint_as_float(r[i + 0]), __uint_as_float(r[i + 1]));
                             pk.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
@@ -152,7 +147,8 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+    cluster_sync();                                           // the partner is done with this CTA's memory too
+    if (warp == 0) tmem_dealloc_pair(tmem, kTmemCols);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -204,7 +200,7 @@ extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_
     }
     if (M == 0) return PEC_OK;
     CUtensorMap tm_x, tm_w;
-    if (!lin::make_map(&tm_x, x, M, K, x_stride, lin::kBM) || !lin::make_map(&tm_w, w, N, K, w_stride, lin::kBN)) {
+    if (!lin::make_map(&tm_x, x, M, K, x_stride, lin::kBM) || !lin::make_map(&tm_w, w, N, K, w_stride, 128)) {
         set_error("pec_linear: cuTensorMapEncodeTiled failed");
         return PEC_ERR_CUDA;
     }
@@ -212,9 +208,9 @@ extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_
         set_error("pec_linear: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
         return PEC_ERR_CUDA;
     }
-    const int64_t gm = (M + lin::kBM - 1) / lin::kBM, gn = (N + lin::kBN - 1) / lin::kBN;
+    const int64_t pairs = (M + 2 * lin::kBM - 1) / (2 * lin::kBM), gn = (N + lin::kBN - 1) / lin::kBN;
     if (gn > 65535) { set_error("pec_linear: N too large"); return PEC_ERR_UNSUPPORTED; }
-    dim3 grid((unsigned)gm, (unsigned)gn);
+    dim3 grid((unsigned)(2 * pairs), (unsigned)gn);           // clusters of two CTAs along x
     lin::linear_kernel<<<grid, lin::kThreads, lin::kSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(
         tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, status);
     const cudaError_t err = cudaGetLastError();
