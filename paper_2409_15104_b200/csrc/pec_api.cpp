@@ -127,7 +127,8 @@ extern "C" int pec_prefill_attn(const pec_attn_args *args, void *cuda_stream)
     if (rc != PEC_OK) return rc;
     if (p.total_rows == 0) return PEC_OK;   // nothing to write
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    return args->in_dtype == PEC_BF16 ? launch_attn_bf16(p, stream) : launch_attn_f32(p, stream);
+    if (args->in_dtype != PEC_BF16) return launch_attn_f32(p, stream);
+    return launch_attn_prefill_bf16(p, stream);
 }
 
 extern "C" int pec_attn_merge(const void *o_a, const float *lse_a, const void *o_b, const float *lse_b,

@@ -1,0 +1,518 @@
+// bf16 partial causal attention on the sm_100a tensor cores (Eq. 3-4 as KV-tile partial attention
+// with online-softmax state: running max, running sum, fp32 accumulator) - the kernel behind
+// pec_prefill_attn for every launch that is not split over the keys.
+//
+// One CTA = one head x 256 query rows, handled as two 128-row tiles ("stages").  Warp roles (three
+// warpgroups):
+//   warps 0-3   softmax of stage 0 (one query row per thread = one TMEM lane)
+//   warps 4-7   softmax of stage 1
+//   warp  8, 10 MMA issuers of stage 0 and stage 1 (one elected lane issues the stage's tcgen05.mma)
+//   warp  9     TMA loader (Q once, then K and V tiles through a ring of shared-memory slots)
+//   warp  11    idle; it completes the third warpgroup so that it can hand its registers to the
+//               softmax warpgroups (setmaxnreg acts on whole warpgroups)
+// K and V arrive as 128-key tiles, but scores are produced and consumed in halves of 64 keys: each
+// stage owns two 64-column score buffers in tensor memory, and half h uses buffer h & 1.
+// S(h) = Q K_h^T lands in its buffer, the softmax warps turn it into P(h) (bf16, written over the
+// first 32 columns of the same buffer), and O += P(h) V_h accumulates in tensor memory.  S(h+1)
+// sits in the other buffer, so it is issued before the softmax of half h is done; per stage the
+// issue order is
+//   PV(h), S(h+2), PV(h+1), S(h+3), ...
+// interleaved between the two stages: a stage's softmax finds its next scores waiting, and the
+// tensor pipe has the other buffer's and the other stage's work queued.  The accumulator is
+// rescaled lazily: the reference maximum of a row only moves when the new maximum exceeds it by
+// 2^8, and a warp that has to rescale first waits for the PV product still in flight on its O.
+//
+// TMEM columns: stage s scores [128 s, 128 s + 128) as two buffers of 64; O_s [256 + 128 s, +128).
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include "pec_internal.h"
+#include "pec_sm100.cuh"
+#include "pec_tile.cuh"
+
+namespace pec {
+using namespace sm100;
+namespace pf {
+
+constexpr int kTile = 128;                                 // rows per stage, keys per K/V tile
+constexpr int kHalf = 64;                                  // keys per score buffer
+constexpr int kBlockM = 2 * kTile;                         // query rows per CTA
+constexpr int kStages = 4;                                 // K/V ring slots
+constexpr int kThreads = 384;                              // three full warpgroups
+constexpr int kSoftmaxWarps = 8, kMmaWarp0 = 8, kLoadWarp = 9, kMmaWarp1 = 10;
+constexpr int kLightRegs = 56, kSoftmaxRegs = 224;          // 256 * 224 + 128 * 56 = 384 * 168 (the launch allocation)
+constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;          // one TMA box: 128 rows x 64 channels
+constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;        // 128 x 128 bf16
+constexpr uint32_t kKeyHalfBytes = kHalf * 128;            // 64 rows of a box (128 bytes per row)
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256;                 // + 128 * stage
+constexpr float kRescaleThreshold = 8.0f;                  // log2 units
+constexpr long long kWaitCycles = 2000000000LL;            // bounded waits give up after ~1 s
+constexpr uint32_t kSuspendNs = 2000;                      // a waiting thread sleeps in the barrier unit this long per try
+
+// What a CTA works on, worked out once by thread 0 and shared through shared memory.  All rows and
+// positions fit in 32 bits (the host rejects larger problems).
+struct Geom {
+    int32_t found;               // 0: tile index past the end (or the launch was already aborted)
+    int32_t q_row0, out_row0, kv_row0;
+    int32_t rows[2];             // valid query rows per stage
+    int32_t pos0[2];             // position of each stage's first row in its request
+    int32_t n[2];                // key tiles each stage takes part in (a prefix of the CTA's walk)
+    int32_t lo[2], hi[2];        // visible-key intervals (positions)
+    int32_t cnt[2];              // key tiles per interval walked by the CTA (union over both stages)
+    int32_t n_max;               // cnt[0] + cnt[1]
+};
+
+struct Shared {
+    uint64_t bar_q;
+    uint64_t kv_full[kStages], kv_empty[kStages];
+    uint64_t s_full[2][2], p_ready[2][2];   // [stage][buffer]
+    uint64_t pv_done[2];                     // one phase per PV product of the stage
+    uint64_t o_final[2];                     // the stage's last PV product is done
+    Geom g;
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+constexpr size_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*alignment slack*/ + sizeof(Shared);
+
+// Bounded mbarrier wait.  Returns false (and raises the abort flag / status word) on expiry.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *sh, int32_t *status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait_suspend(bar, parity, kSuspendNs)) {
+        if (sh->abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            sh->abort_flag = 1;
+            if (status) atomicExch(status, (int)PEC_ERR_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                         const __grid_constant__ CUtensorMap tm_v, const AttnParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
+    const uint32_t sQ = tiles, sRing = tiles + 2 * kTileBytes;
+    Shared *sh = reinterpret_cast<Shared *>(smem_raw + (tiles - raw) + (2 + kStages) * kTileBytes);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int h = blockIdx.y, kvh = h / p.group;
+
+    // Thread 0 works out the CTA's geometry: heaviest (latest) causal tiles first; per stage the
+    // rows, positions and number of key tiles it takes part in.  Key tiles are walked interval 0
+    // first, then interval 1, in ascending position, so each stage's tiles are a prefix of the walk.
+    if (tid == 0) {
+        Geom g;
+        TileJob job;
+        g.found = locate_tile(p, (int64_t)gridDim.x - 1 - blockIdx.x, kBlockM, job) ? 1 : 0;
+        // An earlier CTA's wait expired: the launch is already lost, leave at once.
+        if (p.status && *reinterpret_cast<volatile int32_t *>(p.status) != 0) g.found = 0;
+        sh->abort_flag = 0;
+        if (g.found) {
+            g.q_row0 = (int32_t)job.q_row0; g.out_row0 = (int32_t)job.out_row0; g.kv_row0 = (int32_t)job.kv_row0;
+            g.cnt[0] = g.cnt[1] = 0;
+            for (int t = 0; t < 2; ++t) { g.lo[t] = (int32_t)job.iv_lo[t]; g.hi[t] = (int32_t)job.iv_hi[t]; }
+            for (int st = 0; st < 2; ++st) {
+                int32_t rows = job.n_rows - st * kTile;
+                rows = rows < 0 ? 0 : (rows > kTile ? kTile : rows);
+                g.rows[st] = rows;
+                g.pos0[st] = (int32_t)job.q_pos0 + st * kTile;
+                g.n[st] = 0;
+                if (rows > 0) {
+                    const int32_t last = g.pos0[st] + rows - 1;
+                    for (int t = 0; t < job.n_iv; ++t) {
+                        int32_t end = g.hi[t];
+                        if (p.causal && end > last + 1) end = last + 1;
+                        const int32_t c = end > g.lo[t] ? (end - g.lo[t] + kTile - 1) / kTile : 0;
+                        g.n[st] += c;
+                        g.cnt[t] = c > g.cnt[t] ? c : g.cnt[t];
+                    }
+                }
+            }
+            g.n_max = g.cnt[0] + g.cnt[1];
+        }
+        sh->g = g;
+    }
+    __syncthreads();
+    if (!sh->g.found) return;
+    const int n_max = sh->g.n_max;
+
+    if (tid == 0) {
+        mbar_init(smem_u32(&sh->bar_q), 1);
+        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->kv_full[s]), 1); mbar_init(smem_u32(&sh->kv_empty[s]), 2); }
+        for (int st = 0; st < 2; ++st) {
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(smem_u32(&sh->s_full[st][b]), 1);
+                mbar_init(smem_u32(&sh->p_ready[st][b]), 4);  // one arrival per softmax warp
+            }
+            mbar_init(smem_u32(&sh->pv_done[st]), 1);
+            mbar_init(smem_u32(&sh->o_final[st]), 1);
+        }
+        mbar_init_fence();
+        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_alloc(smem_u32(&sh->tmem_base), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh->tmem_base;
+
+    // Warps 8-11 (the whole third warpgroup) give registers up, warps 0-7 take them.
+    if (warp == kLoadWarp) {
+        // ------------------------------------------------------------------ TMA loader
+        reg_dealloc<kLightRegs>();
+        if (lane == 0 && n_max > 0) {
+            const uint32_t bar_q = smem_u32(&sh->bar_q);
+            mbar_arrive_expect_tx(bar_q, 2 * kTileBytes);
+#pragma unroll
+            for (int st = 0; st < 2; ++st) {
+                const int row = sh->g.q_row0 + st * kTile;
+                tma_load_3d(sQ + st * kTileBytes, &tm_q, bar_q, 0, h, row);
+                tma_load_3d(sQ + st * kTileBytes + kHalfTileBytes, &tm_q, bar_q, 64, h, row);
+            }
+            for (int i = 0; i < 2 * n_max; ++i) {              // items: K(0), V(0), K(1), V(1), ...
+                const int slot = i % kStages, fill = i / kStages;
+                if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p.status)) break;
+                const int jt = i >> 1, c0 = sh->g.cnt[0];
+                const int krow = sh->g.kv_row0 + (jt < c0 ? sh->g.lo[0] + jt * kTile : sh->g.lo[1] + (jt - c0) * kTile);
+                const void *map = (i & 1) ? (const void *)&tm_v : (const void *)&tm_k;
+                const uint32_t dst = sRing + slot * kTileBytes, bar = smem_u32(&sh->kv_full[slot]);
+                mbar_arrive_expect_tx(bar, kTileBytes);
+                tma_load_3d(dst, map, bar, 0, kvh, krow);
+                tma_load_3d(dst + kHalfTileBytes, map, bar, 64, kvh, krow);
+            }
+        }
+        __syncwarp();
+    } else if (warp == kMmaWarp0 || warp == kMmaWarp1) {
+        // ------------------------------------------------------------------ MMA issuers, one warp per stage
+        // The whole warp walks the loop and one elected lane issues: addresses, descriptors and loop
+        // state stay warp-uniform, which keeps the instruction count per MMA low.  An issuer shares its
+        // scheduler with two softmax warps, and one warp issuing for both stages was the kernel's
+        // bottleneck; the two stages touch disjoint tensor memory, so their MMAs need no order between
+        // them.  Each issuer waits for and releases every ring item, used by its stage or not, so the
+        // "empty" barriers always see two arrivals per item.
+        reg_dealloc<kLightRegs>();
+        if (n_max > 0) {
+            const int st = (warp == kMmaWarp0) ? 0 : 1;
+            const bool leader = elect_one();
+            constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kHalf, 0, 0);
+            constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, kHeadDim, 0, 1);
+            auto wait_u = [&](uint64_t *bar, uint32_t parity) {
+                return __all_sync(0xffffffffu, wait_bar(smem_u32(bar), parity, sh, p.status));
+            };
+            auto kv_wait = [&](int item) { return wait_u(&sh->kv_full[item % kStages], (item / kStages) & 1); };
+            auto kv_release = [&](int item) { if (leader) tc_commit(smem_u32(&sh->kv_empty[item % kStages])); };
+            const uint32_t a_lo = desc_lo(sQ + st * kTileBytes, 16);
+            const uint32_t tS = tmem + kColS + st * kTile, tO = tmem + kColO + st * kTile;
+            // S(hf) = Q K^T for the 64 keys of half hf (tile hf / 2, rows 64 (hf & 1) .. of it): both operands
+            // K-major; 8 steps of 16 channels, 4 per 64-channel box; the half's rows start 8 KiB into each box.
+            auto issue_qk = [&](int hf) {
+                const int item = 2 * (hf >> 1), b = hf & 1;
+                const uint32_t k_lo = desc_lo(sRing + (item % kStages) * kTileBytes + b * kKeyHalfBytes, 16);
+                if (leader) {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        constexpr uint32_t kBox = kHalfTileBytes >> 4;
+                        const uint32_t off = (uint32_t)(ks >> 2) * kBox + (uint32_t)(ks & 3) * 2u;   // 32 bytes per K step, in 16-byte units
+                        mma_ss_lh(tS + b * kHalf, a_lo + off, k_lo + off, idesc_qk, ks > 0 ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&sh->s_full[st][b]));
+                }
+            };
+            // O (+)= P(hf) V: A = P from TMEM (8 columns per 16 keys), B = the half's 64 keys of the V tile
+            // stored [key][channel] (N-contiguous): 16 keys = 2048 bytes per step, channel halves 16 KiB apart.
+            auto issue_pv = [&](int hf, bool last) {
+                const int item = 2 * (hf >> 1) + 1, b = hf & 1;
+                const uint32_t v_lo = desc_lo(sRing + (item % kStages) * kTileBytes + b * kKeyHalfBytes, kHalfTileBytes);
+                if (leader) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        mma_ts_lh(tO, tS + b * kHalf + ks * 8, v_lo + ks * (2048u >> 4), idesc_pv, (hf > 0 || ks > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&sh->pv_done[st]));
+                    if (last) tc_commit(smem_u32(&sh->o_final[st]));
+                }
+            };
+
+            const int n_hf = 2 * sh->g.n[st];                  // halves of this stage
+            bool ok = wait_u(&sh->bar_q, 0) && kv_wait(0);
+            if (ok) {
+                if (n_hf > 0) { issue_qk(0); issue_qk(1); }
+                kv_release(0);
+            }
+            for (int hf = 0; hf < 2 * n_max && ok; ++hf) {
+                const int j = hf >> 1, b = hf & 1;
+                const bool has_next = j + 1 < n_max;
+                if (b == 0) ok = kv_wait(2 * j + 1);           // V(j)
+                if (ok && hf < n_hf) {
+                    ok = wait_u(&sh->p_ready[st][b], j & 1);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(hf, hf == n_hf - 1);
+                }
+                if (ok && b == 0 && has_next) ok = kv_wait(2 * j + 2);   // K(j+1)
+                if (!ok) break;
+                if (hf + 2 < n_hf) issue_qk(hf + 2);
+                if (b == 1) {
+                    kv_release(2 * j + 1);
+                    if (has_next) kv_release(2 * j + 2);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp >= kSoftmaxWarps) {
+        reg_dealloc<kLightRegs>();
+    } else {
+        // ------------------------------------------------------------------ softmax + epilogue
+        reg_alloc<kSoftmaxRegs>();
+        const int st = warp >> 2, quarter = warp & 3;
+        const int row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+        const uint32_t tS = tmem + lane_base + kColS + st * kTile;
+        const uint32_t tO = tmem + lane_base + kColO + st * kTile;
+        const int n_hf = 2 * sh->g.n[st];
+        const uint32_t bar_pv = smem_u32(&sh->pv_done[st]);
+        // Per interval: where it ends, and the first key position that some row of this stage cannot
+        // see (halves reaching past it need the mask).
+        const int pos0 = sh->g.pos0[st], my_pos = pos0 + row_in_tile, hf0 = 2 * sh->g.cnt[0];
+        int iv_full[2], iv_mine[2];
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const int hi_t = sh->g.hi[t];
+            iv_full[t] = (p.causal && pos0 + 1 < hi_t) ? pos0 + 1 : hi_t;
+            iv_mine[t] = (p.causal && my_pos + 1 < hi_t) ? my_pos + 1 : hi_t;
+        }
+        int k0 = sh->g.lo[0], cur = 0;
+
+        float m_ref = -INFINITY, l_run = 0.f;                // m_ref in log2 units of the scaled scores
+        bool ok = true;
+        // The special-function unit is the softmax's bottleneck and this warp shares its scheduler's
+        // unit with the warp of the other stage that has the same quarter.  The two take turns at the
+        // exponentials of a half (a token passed through two named barriers), so one warp's loads,
+        // maxima and stores run under the other's exponentials instead of both phases colliding.
+        // The turns cover the halves both stages have; a warp whose wait failed keeps passing the
+        // token (and does nothing else) so that its partner never blocks on it.
+        const int n_turns = 2 * (sh->g.n[0] < sh->g.n[1] ? sh->g.n[0] : sh->g.n[1]);
+        const uint32_t tok_mine = 1 + 2 * quarter + st, tok_other = 1 + 2 * quarter + (st ^ 1);
+        if (st == 1 && n_turns > 0) named_arrive64(tok_other);   // stage 0 goes first
+        for (int hf = 0; hf < n_hf; ++hf, k0 += kHalf) {
+            if (hf == hf0) { cur = 1; k0 = sh->g.lo[1]; }
+            const int b = hf & 1;
+            const bool turn = hf < n_turns;
+            uint32_t r[kHalf];
+            float2 sc2, nm2;
+            if (ok) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->s_full[st][b]), (hf >> 1) & 1, sh, p.status));   // warp-uniform
+            if (ok) {
+                tc_fence_after();
+                tmem_ld64(tS + b * kHalf, r);
+                // Mask only when some row of this stage cannot see the whole half.
+                const bool masked = k0 + kHalf > (cur ? iv_full[1] : iv_full[0]);
+                if (masked) {
+                    int n_vis = (cur ? iv_mine[1] : iv_mine[0]) - k0;
+                    n_vis = n_vis < 0 ? 0 : (n_vis > kHalf ? kHalf : n_vis);
+#pragma unroll
+                    for (int c = 0; c < kHalf; ++c) r[c] = (c < n_vis) ? r[c] : 0xff800000u;   // -inf
+                }
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < kHalf; c += 8) {
+                    mx0 = fmax3(mx0, __uint_as_float(r[c + 0]), __uint_as_float(r[c + 1]));
+                    mx1 = fmax3(mx1, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+                    mx2 = fmax3(mx2, __uint_as_float(r[c + 4]), __uint_as_float(r[c + 5]));
+                    mx3 = fmax3(mx3, __uint_as_float(r[c + 6]), __uint_as_float(r[c + 7]));
+                }
+                const float m_new = fmax3(mx0, mx1, fmaxf(mx2, mx3)) * p.scale_log2;   // -inf stays -inf (scale > 0)
+
+                // Lazy rescale: move the reference maximum only when it is outgrown by 2^8.
+                float alpha = 1.f;
+                const bool grow = m_new > m_ref + kRescaleThreshold;
+                if (grow) {
+                    alpha = ex2(m_ref - m_new);                   // 0 when the row had no key so far
+                    m_ref = m_new;
+                    l_run *= alpha;
+                }
+                if (hf > 0 && __any_sync(0xffffffffu, grow)) {
+                    // O still receives P(hf-1) V: wait for that product (phase hf-1 of the stage's PV barrier;
+                    // PV(hf) cannot be issued before this warp hands P(hf) over, so the phase is unambiguous).
+                    ok = __all_sync(0xffffffffu, wait_bar(bar_pv, (hf - 1) & 1, sh, p.status));
+                    if (ok) {
+                        tc_fence_after();
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c * 32, o);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st32(tO + c * 32, o);
+                        }
+                    }
+                }
+                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+                sc2 = make_float2(p.scale_log2, p.scale_log2);
+                nm2 = make_float2(neg_m, neg_m);
+            }
+            if (turn) named_sync64(tok_mine);
+            if (ok) {
+                float2 sum[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sum[i] = make_float2(0.f, 0.f);
+                // p = 2^(s * scale - m): packed FMA for the argument, the special-function unit for 2^x, packed
+                // adds for the row sum.  P is packed to bf16 pairs: column c of the A operand holds keys 2c (low
+                // half) and 2c+1 (high half); r[i] is reused for pair i.
+#pragma unroll
+                for (int i = 0; i < kHalf / 2; ++i) {
+                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, nm2);
+                    const float2 e = make_float2(ex2(x.x), ex2(x.y));
+                    sum[i & 3] = __fadd2_rn(sum[i & 3], e);
+                    r[i] = pack_bf16(e.x, e.y);
+                }
+                const float2 s01 = __fadd2_rn(__fadd2_rn(sum[0], sum[1]), __fadd2_rn(sum[2], sum[3]));
+                l_run += s01.x + s01.y;
+            }
+            if (turn && !(st == 1 && hf == n_turns - 1)) named_arrive64(tok_other);
+            if (ok) {
+                tmem_st32(tS + b * kHalf, r);
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sh->p_ready[st][b]));
+            }
+        }
+
+        // Epilogue: O / l and LSE = ln2 * m + ln l; rows without any visible key give 0 and -inf.
+        if (ok && n_hf > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->o_final[st]), 0, sh, p.status));
+        if (ok && sh->g.rows[st] > 0) {
+            tc_fence_after();
+            const bool valid = row_in_tile < sh->g.rows[st];
+            const bool empty = (l_run == 0.f);
+            const float inv = empty ? 0.f : 1.f / l_run;
+            const int64_t row = (int64_t)sh->g.out_row0 + st * kTile + row_in_tile;
+            const int64_t obase = (row * p.Hq + h) * kHeadDim;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                if (n_hf == 0) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;
+                } else {
+                    tmem_ld32(tO + c * 32, r);                // warp-wide; only the stores are predicated
+                }
+                if (!valid) continue;
+                if (p.o_is_bf16) {
+                    __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(p.o) + obase + c * 32;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 pk;
+                        pk.x = pack_bf16(__uint_as_float(r[i + 0]) * inv, __uint_as_float(r[i + 1]) * inv);
+                        pk.y = pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+                        pk.z = pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
+                        pk.w = pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(o + i) = pk;
+                    }
+                } else {
+                    float *o = static_cast<float *>(p.o) + obase + c * 32;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4)
+                        *reinterpret_cast<float4 *>(o + i) = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
+                                                                         __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+                }
+            }
+            if (valid) p.lse[row * p.Hq + h] = empty ? -INFINITY : m_ref * 0.6931471805599453f + logf(l_run);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+// ------------------------------------------------------------------------------------------ host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// [rows, heads, 128] bf16 tensor with element strides (stride_t, stride_h); box = 64 channels x 1 head x 128 rows.
+static bool make_map(CUtensorMap *map, const void *base, int64_t rows, int32_t heads, int64_t stride_t, int64_t stride_h)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)heads, (cuuint64_t)(rows > 0 ? rows : 1)};
+    cuuint64_t strides[2] = {(cuuint64_t)stride_h * 2, (cuuint64_t)stride_t * 2};
+    cuuint32_t box[3] = {64, 1, 128};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace pf
+
+int launch_attn_prefill_bf16(const AttnParams &p, cudaStream_t stream)
+{
+    using namespace pf;
+    if (!p.status) { set_error("pec_prefill_attn: the bf16 path needs a status word"); return PEC_ERR_INVALID_ARG; }
+    if (p.splits != 1) { set_error("pec_prefill_attn: this kernel takes no split launches"); return PEC_ERR_INVALID_ARG; }
+    // Rows the maps may touch: queries up to the chunk end, keys up to the end of the visible subset.
+    int64_t q_rows, kv_rows;
+    if (p.cu_seqlens) { q_rows = p.total_rows; kv_rows = p.total_rows; }
+    else {
+        q_rows = p.chunk_start + p.chunk_len;
+        kv_rows = 0;
+        for (int t = 0; t < p.n_iv; ++t) kv_rows = p.iv_hi[t] > kv_rows ? p.iv_hi[t] : kv_rows;
+    }
+    if (q_rows >= ((int64_t)1 << 31) || kv_rows >= ((int64_t)1 << 31)) {
+        set_error("pec_prefill_attn: more than 2^31 rows unsupported");
+        return PEC_ERR_UNSUPPORTED;
+    }
+    CUtensorMap tm_q, tm_k, tm_v;
+    if (!make_map(&tm_q, p.q, q_rows, p.Hq, p.q_stride_t, p.q_stride_h) ||
+        !make_map(&tm_k, p.k, kv_rows, p.Hkv, p.k_stride_t, p.k_stride_h) ||
+        !make_map(&tm_v, p.v, kv_rows, p.Hkv, p.v_stride_t, p.v_stride_h)) {
+        set_error("pec_prefill_attn: cuTensorMapEncodeTiled failed (driver too old, or strides/addresses not encodable)");
+        return PEC_ERR_CUDA;
+    }
+    if (cudaFuncSetAttribute(attn_prefill_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) {
+        set_error("pec_prefill_attn: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
+        return PEC_ERR_CUDA;
+    }
+    // The softmax warpgroups take registers the third warpgroup gives up; that only works when the
+    // launch allocation (registers per thread x threads) covers the new split.
+    cudaFuncAttributes attr;
+    if (cudaFuncGetAttributes(&attr, attn_prefill_bf16_kernel) != cudaSuccess ||
+        attr.numRegs * kThreads < kSoftmaxWarps * 32 * kSoftmaxRegs + (kThreads - kSoftmaxWarps * 32) * kLightRegs) {
+        set_error("pec_prefill_attn: kernel register allocation too small for the warp-role register split");
+        return PEC_ERR_CUDA;
+    }
+    int64_t tiles = (p.total_rows + kBlockM - 1) / kBlockM;
+    if (p.cu_seqlens) tiles += p.B;
+    if (tiles > 0x7fffffff || p.Hq > 65535) { set_error("pec_prefill_attn: grid too large"); return PEC_ERR_UNSUPPORTED; }
+    dim3 grid((unsigned)tiles, (unsigned)p.Hq, 1);
+    attn_prefill_bf16_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, p);
+    const cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) { set_error("pec_prefill_attn: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
+    return PEC_OK;
+}
+
+}  // namespace pec
