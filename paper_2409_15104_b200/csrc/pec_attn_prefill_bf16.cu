@@ -53,7 +53,7 @@ constexpr uint32_t kSuspendNs = 2000;                      // a waiting thread s
 // What a CTA works on, worked out once by thread 0 and shared through shared memory.  All rows and
 // positions fit in 32 bits (the host rejects larger problems).
 struct Geom {
-    int32_t found;               // 0: tile index past the end (or the launch was already aborted)
+    int32_t found;               // 0: tile index past the end
     int32_t q_row0, out_row0, kv_row0;
     int32_t rows[2];             // valid query rows per stage
     int32_t pos0[2];             // position of each stage's first row in its request
@@ -107,12 +107,12 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     // Thread 0 works out the CTA's geometry: heaviest (latest) causal tiles first; per stage the
     // rows, positions and number of key tiles it takes part in.  Key tiles are walked interval 0
     // first, then interval 1, in ascending position, so each stage's tiles are a prefix of the walk.
+    // The set-up runs in parallel: warp 1 initialises the barriers and prefetches the tensor maps,
+    // warp 2 allocates tensor memory, thread 0 works out the geometry.
     if (tid == 0) {
-        Geom g;
+        Geom g = {};
         TileJob job;
         g.found = locate_tile(p, (int64_t)gridDim.x - 1 - blockIdx.x, kBlockM, job) ? 1 : 0;
-        // An earlier CTA's wait expired: the launch is already lost, leave at once.
-        if (p.status && *reinterpret_cast<volatile int32_t *>(p.status) != 0) g.found = 0;
         sh->abort_flag = 0;
         if (g.found) {
             g.q_row0 = (int32_t)job.q_row0; g.out_row0 = (int32_t)job.out_row0; g.kv_row0 = (int32_t)job.kv_row0;
@@ -137,13 +137,9 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             }
             g.n_max = g.cnt[0] + g.cnt[1];
         }
-        sh->g = g;
-    }
-    __syncthreads();
-    if (!sh->g.found) return;
-    const int n_max = sh->g.n_max;
-
-    if (tid == 0) {
+        sh->g = g;                                            // a CTA past the last tile has no rows and no keys
+    } else if (tid == 32) {
+        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
         mbar_init(smem_u32(&sh->bar_q), 1);
         for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->kv_full[s]), 1); mbar_init(smem_u32(&sh->kv_empty[s]), 2); }
         for (int st = 0; st < 2; ++st) {
@@ -155,16 +151,14 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             mbar_init(smem_u32(&sh->o_final[st]), 1);
         }
         mbar_init_fence();
-        prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
-    }
-    if (warp == 0) {
-        __syncwarp();
+    } else if (warp == 2) {
         tmem_alloc(smem_u32(&sh->tmem_base), kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    const int n_max = sh->g.n_max;
     const uint32_t tmem = sh->tmem_base;
 
     // Warps 8-11 (the whole third warpgroup) give registers up, warps 0-7 take them.
@@ -182,6 +176,7 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             }
             for (int i = 0; i < 2 * n_max; ++i) {              // items: K(0), V(0), K(1), V(1), ...
                 const int slot = i % kStages, fill = i / kStages;
+                if (sh->abort_flag) break;
                 if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p.status)) break;
                 const int jt = i >> 1, c0 = sh->g.cnt[0];
                 const int krow = sh->g.kv_row0 + (jt < c0 ? sh->g.lo[0] + jt * kTile : sh->g.lo[1] + (jt - c0) * kTile);
@@ -212,32 +207,29 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             };
             auto kv_wait = [&](int item) { return wait_u(&sh->kv_full[item % kStages], (item / kStages) & 1); };
             auto kv_release = [&](int item) { if (leader) tc_commit(smem_u32(&sh->kv_empty[item % kStages])); };
-            const uint32_t a_lo = desc_lo(sQ + st * kTileBytes, 16);
             const uint32_t tS = tmem + kColS + st * kTile, tO = tmem + kColO + st * kTile;
+            // Descriptors: the stage's Q tile gives eight fixed A descriptors (16 channels per K step, four steps
+            // per 64-channel box); a K or V half is the ring's first descriptor plus slot and half offsets.
+            constexpr uint32_t kBox16 = kHalfTileBytes >> 4;
+            uint64_t a_desc[8];
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+                a_desc[ks] = smem_desc_sw128(sQ + st * kTileBytes + (uint32_t)(ks >> 2) * kHalfTileBytes + (uint32_t)(ks & 3) * 32u, 16, 1024);
+            const uint64_t k_ring = smem_desc_sw128(sRing, 16, 1024), v_ring = smem_desc_sw128(sRing, kHalfTileBytes, 1024);
             // S(hf) = Q K^T for the 64 keys of half hf (tile hf / 2, rows 64 (hf & 1) .. of it): both operands
-            // K-major; 8 steps of 16 channels, 4 per 64-channel box; the half's rows start 8 KiB into each box.
+            // K-major; the half's rows start 8 KiB into each box.
             auto issue_qk = [&](int hf) {
                 const int item = 2 * (hf >> 1), b = hf & 1;
-                const uint32_t k_lo = desc_lo(sRing + (item % kStages) * kTileBytes + b * kKeyHalfBytes, 16);
-                if (leader) {
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        constexpr uint32_t kBox = kHalfTileBytes >> 4;
-                        const uint32_t off = (uint32_t)(ks >> 2) * kBox + (uint32_t)(ks & 3) * 2u;   // 32 bytes per K step, in 16-byte units
-                        mma_ss_lh(tS + b * kHalf, a_lo + off, k_lo + off, idesc_qk, ks > 0 ? 1u : 0u);
-                    }
-                    tc_commit(smem_u32(&sh->s_full[st][b]));
-                }
+                const uint64_t k0 = k_ring + (uint32_t)(((item % kStages) * kTileBytes + b * kKeyHalfBytes) >> 4);
+                if (leader) mma_ss_k128_commit<kBox16>(tS + b * kHalf, a_desc, k0, idesc_qk, smem_u32(&sh->s_full[st][b]));
             };
             // O (+)= P(hf) V: A = P from TMEM (8 columns per 16 keys), B = the half's 64 keys of the V tile
             // stored [key][channel] (N-contiguous): 16 keys = 2048 bytes per step, channel halves 16 KiB apart.
             auto issue_pv = [&](int hf, bool last) {
                 const int item = 2 * (hf >> 1) + 1, b = hf & 1;
-                const uint32_t v_lo = desc_lo(sRing + (item % kStages) * kTileBytes + b * kKeyHalfBytes, kHalfTileBytes);
+                const uint64_t v0 = v_ring + (uint32_t)(((item % kStages) * kTileBytes + b * kKeyHalfBytes) >> 4);
                 if (leader) {
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        mma_ts_lh(tO, tS + b * kHalf + ks * 8, v_lo + ks * (2048u >> 4), idesc_pv, (hf > 0 || ks > 0) ? 1u : 0u);
+                    mma_ts_k64(tO, tS + b * kHalf, v0, idesc_pv, hf > 0 ? 1u : 0u);
                     tc_commit(smem_u32(&sh->pv_done[st]));
                     if (last) tc_commit(smem_u32(&sh->o_final[st]));
                 }
@@ -270,7 +262,11 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         }
         __syncwarp();
     } else if (warp >= kSoftmaxWarps) {
+        // The spare warp looks at the caller's status word: if an earlier CTA's wait expired the launch is
+        // lost, and raising the abort flag stops the loader, after which every wait of this CTA fails fast.
+        // (Kept off the start-up path: the word is a global-memory read.)
         reg_dealloc<kLightRegs>();
+        if (lane == 0 && p.status && *reinterpret_cast<volatile int32_t *>(p.status) != 0) sh->abort_flag = 1;
     } else {
         // ------------------------------------------------------------------ softmax + epilogue
         reg_alloc<kSoftmaxRegs>();
@@ -389,50 +385,72 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         }
 
         // Epilogue: O / l and LSE = ln2 * m + ln l; rows without any visible key give 0 and -inf.
+        // A thread holds one whole row, so storing from registers would touch 32 rows per instruction.
+        // Each warp instead stages 32 rows x 256 bytes in its quarter of the stage's Q tile (no longer
+        // read once the stage's last product is done; 16-byte chunks XOR-swizzled by row against bank
+        // conflicts) and writes it out two rows per instruction, 256 contiguous bytes each.
         if (ok && n_hf > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->o_final[st]), 0, sh, p.status));
+        // A stage without keys never waited for its Q tile: the load must have landed before the tile is reused.
+        if (ok && n_hf == 0 && n_max > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->bar_q), 0, sh, p.status));
         if (ok && sh->g.rows[st] > 0) {
             tc_fence_after();
-            const bool valid = row_in_tile < sh->g.rows[st];
             const bool empty = (l_run == 0.f);
             const float inv = empty ? 0.f : 1.f / l_run;
-            const int64_t row = (int64_t)sh->g.out_row0 + st * kTile + row_in_tile;
-            const int64_t obase = (row * p.Hq + h) * kHeadDim;
+            const int rows_valid = sh->g.rows[st] - quarter * 32;                 // of this warp's 32 rows
+            const int64_t row0 = (int64_t)sh->g.out_row0 + st * kTile + quarter * 32;
+            uint8_t *stage_buf = smem_raw + (tiles - raw) + st * kTileBytes + quarter * 8192;
+            uint8_t *my_row = stage_buf + lane * 256;
+            const int sub = lane >> 4, chunk = lane & 15;                        // read-back: row parity and 16-byte chunk
+            const int n_pass = p.o_is_bf16 ? 1 : 2;                              // 256 bytes of a row per pass
+            for (int pass = 0; pass < n_pass; ++pass) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                if (n_hf == 0) {
+                for (int c = 0; c < 4; ++c) {
+                    if (!p.o_is_bf16 && (c >> 1) != pass) continue;
+                    uint32_t r[32];
+                    if (n_hf == 0) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = 0u;
-                } else {
-                    tmem_ld32(tO + c * 32, r);                // warp-wide; only the stores are predicated
-                }
-                if (!valid) continue;
-                if (p.o_is_bf16) {
-                    __nv_bfloat16 *o = static_cast<__nv_bfloat16 *>(p.o) + obase + c * 32;
-#pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        uint4 pk;
-                        pk.x = pack_bf16(__uint_as_float(r[i + 0]) * inv, __uint_as_float(r[i + 1]) * inv);
-                        pk.y = pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-                        pk.z = pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
-                        pk.w = pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(o + i) = pk;
+                        for (int i = 0; i < 32; ++i) r[i] = 0u;
+                    } else {
+                        tmem_ld32(tO + c * 32, r);
                     }
-                } else {
-                    float *o = static_cast<float *>(p.o) + obase + c * 32;
+                    if (p.o_is_bf16) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        *reinterpret_cast<float4 *>(o + i) = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
-                                                                         __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+                        for (int i = 0; i < 4; ++i) {                             // 8 channels = 16 bytes per chunk
+                            uint4 pk;
+                            pk.x = pack_bf16(__uint_as_float(r[8 * i + 0]) * inv, __uint_as_float(r[8 * i + 1]) * inv);
+                            pk.y = pack_bf16(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
+                            pk.z = pack_bf16(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv);
+                            pk.w = pack_bf16(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv);
+                            *reinterpret_cast<uint4 *>(my_row + (((c * 4 + i) ^ (lane & 15)) << 4)) = pk;
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {                             // 4 channels = 16 bytes per chunk
+                            const float4 f = make_float4(__uint_as_float(r[4 * i]) * inv, __uint_as_float(r[4 * i + 1]) * inv,
+                                                         __uint_as_float(r[4 * i + 2]) * inv, __uint_as_float(r[4 * i + 3]) * inv);
+                            *reinterpret_cast<float4 *>(my_row + ((((c & 1) * 8 + i) ^ (lane & 15)) << 4)) = f;
+                        }
+                    }
                 }
+                __syncwarp();
+                uint8_t *out = static_cast<uint8_t *>(p.o) + (p.o_is_bf16 ? 0 : pass * 256) + chunk * 16;
+                const int64_t row_bytes = (int64_t)p.Hq * kHeadDim * (p.o_is_bf16 ? 2 : 4);
+                const int64_t head_bytes = (int64_t)h * kHeadDim * (p.o_is_bf16 ? 2 : 4);
+#pragma unroll 4
+                for (int rr = 0; rr < 16; ++rr) {
+                    const int row = 2 * rr + sub;
+                    const uint4 val = *reinterpret_cast<const uint4 *>(stage_buf + row * 256 + ((chunk ^ (row & 15)) << 4));
+                    if (row < rows_valid) *reinterpret_cast<uint4 *>(out + (row0 + row) * row_bytes + head_bytes) = val;
+                }
+                __syncwarp();
             }
-            if (valid) p.lse[row * p.Hq + h] = empty ? -INFINITY : m_ref * 0.6931471805599453f + logf(l_run);
+            if (lane < rows_valid) p.lse[(row0 + lane) * p.Hq + h] = empty ? -INFINITY : m_ref * 0.6931471805599453f + logf(l_run);
         }
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 2) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ------------------------------------------------------------------------------------------ host

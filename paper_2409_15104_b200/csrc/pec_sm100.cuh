@@ -203,6 +203,57 @@ __device__ __forceinline__ void mma_ts_lh(uint32_t d_tmem, uint32_t a_tmem, uint
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Eight K steps (16 channels each) of D = A B^T in one statement, for K-major SWIZZLE_128B tiles whose
+// 128 channels lie in two 64-channel boxes `box16` (in 16-byte units) apart: A descriptors are passed
+// ready-made (they do not change while a CTA keeps its A tile), B is its first descriptor plus
+// constants.  The first step overwrites D.  Ends with a commit to `bar`.
+template <uint32_t kBox16>
+__device__ __forceinline__ void mma_ss_k128_commit(uint32_t d_tmem, const uint64_t (&a)[8], uint64_t b0, uint32_t idesc, uint32_t bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred pf, pt;\n\t.reg .b64 db;\n\t"
+        "setp.ne.u32 pf, %0, %0;\n\t"
+        "setp.eq.u32 pt, %0, %0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %9, %10, pf;\n\t"
+        "add.s64 db, %9, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %2, db, %10, pt;\n\t"
+        "add.s64 db, %9, 4;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %3, db, %10, pt;\n\t"
+        "add.s64 db, %9, 6;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %4, db, %10, pt;\n\t"
+        "add.s64 db, %9, %12;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %5, db, %10, pt;\n\t"
+        "add.s64 db, %9, %13;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %6, db, %10, pt;\n\t"
+        "add.s64 db, %9, %14;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %7, db, %10, pt;\n\t"
+        "add.s64 db, %9, %15;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %8, db, %10, pt;\n\t"
+        "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%11];\n\t}"
+        ::"r"(d_tmem), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(a[4]), "l"(a[5]), "l"(a[6]), "l"(a[7]),
+          "l"(b0), "r"(idesc), "r"(bar),
+          "n"(kBox16), "n"(kBox16 + 2), "n"(kBox16 + 4), "n"(kBox16 + 6) : "memory");
+}
+// Four K steps (16 keys each) of D (+)= A B with A in tensor memory (8 columns per step) and B an
+// N-major SWIZZLE_128B tile (2048 bytes per step); `accumulate` = 0 makes the first step overwrite D.
+__device__ __forceinline__ void mma_ts_k64(uint32_t d_tmem, uint32_t a_tmem, uint64_t b0, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p0, pt;\n\t.reg .b64 db;\n\t.reg .b32 ta;\n\t"
+        "setp.ne.u32 p0, %4, 0;\n\t"
+        "setp.eq.u32 pt, %0, %0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p0;\n\t"
+        "add.s64 db, %2, 128;\n\t"
+        "add.u32 ta, %1, 8;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, pt;\n\t"
+        "add.s64 db, %2, 256;\n\t"
+        "add.u32 ta, %1, 16;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, pt;\n\t"
+        "add.s64 db, %2, 384;\n\t"
+        "add.u32 ta, %1, 24;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, pt;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b0), "r"(idesc), "r"(accumulate) : "memory");
+}
 // D[tmem] (+)= A[tmem] * B[smem]
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {
