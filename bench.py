@@ -290,7 +290,7 @@ def run_ours(args, wl):
         "frac_of_measured_bf16_sustained": tflops / world / peaks["bf16_sustained"],
         "attention_only_tflops": attn_tflops,
         "merge": merge,
-        "roofline": {"bound": "tensor", "kernel": "attn_bf16_kernel", "achieved": attn_tflops,
+        "roofline": {"bound": "tensor", "kernel": "attn_prefill_bf16_kernel", "achieved": attn_tflops,
                      "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": attn_tflops / peaks["bf16_sustained"],
                      "traffic": None, "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step)",
                      "frac_of_burst": attn_tflops / peaks["bf16_burst"], "frac_of_nominal": attn_tflops / NOMINAL_BF16_TFLOPS,

@@ -1,8 +1,10 @@
-// bf16 partial causal attention on the sm_100a tensor cores (Eq. 3-4 as KV-tile partial attention
-// with online-softmax state: running max, running sum, fp32 accumulator).
+// bf16 partial attention of a few query rows against a long key range, split over the keys: the
+// kernel behind pec_decode_attn (Eq. 3-4 as KV-tile partial attention with online-softmax state;
+// the partials of the key slices are merged by their LSE afterwards).
 //
-// One CTA = one head x 256 query rows, handled as two 128-row tiles ("stages") that ping-pong on
-// the tensor core.  Warp roles (three warpgroups):
+// One CTA = one group of query heads (up to 128 rows) x two key slices.  Both 128-row "stages" hold
+// the same query rows and each walks its own slice, so a CTA keeps two slices in flight and one
+// slice's softmax runs under the other's MMAs.  Warp roles (three warpgroups):
 //   warps 0-3   softmax of stage 0 (one query row per thread = one TMEM lane)
 //   warps 4-7   softmax of stage 1
 //   warp  8     MMA issuer (one elected lane issues every tcgen05.mma)
@@ -10,10 +12,9 @@
 //   warps 10-11 idle; they complete the third warpgroup so that it can hand its registers to the
 //               softmax warpgroups (setmaxnreg acts on whole warpgroups)
 // S = Q K^T lands in tensor memory, the softmax warps turn it into P (bf16, written back over the
-// first half of S), and O += P V accumulates in tensor memory; the issue order
-//   PV_0(j), S_0(j+1), PV_1(j), S_1(j+1), ...
-// lets one stage's softmax run under the other stage's two MMAs.  The accumulator is rescaled
-// lazily: the reference maximum of a row only moves when the new maximum exceeds it by 2^8.
+// first half of S), and O += P V accumulates in tensor memory.  The accumulator is rescaled lazily:
+// the reference maximum of a row only moves when the new maximum exceeds it by 2^8.  The kernel is
+// bound by the K/V stream from HBM, not by the tensor pipe.
 //
 // TMEM columns: S_0 [0,128) (P_0 in [0,64)), S_1 [128,256) (P_1 in [128,192)), O_0 [256,384),
 // O_1 [384,512).
@@ -26,6 +27,7 @@
 
 namespace pec {
 using namespace sm100;
+namespace splitk {
 
 constexpr int kTile = 128;                                 // rows per stage, keys per KV tile
 constexpr int kBlockM = 2 * kTile;                         // query rows per CTA
@@ -38,7 +40,6 @@ constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;        // 128 x 128 bf16
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;                 // + 128 * stage
 constexpr float kRescaleThreshold = 8.0f;                  // log2 units
-constexpr int kPolyOf4 = 0;                                // pairs of every 4 whose 2^x runs on the FMA pipe
 constexpr long long kWaitCycles = 2000000000LL;            // bounded waits give up after ~1 s
 constexpr uint32_t kSuspendNs = 2000;                      // a waiting thread sleeps in the barrier unit this long per try
 
@@ -52,13 +53,8 @@ struct Geom {
     int32_t n[2];                // key tiles each stage takes part in (a prefix of the CTA's walk)
     int32_t lo[2], hi[2];        // visible-key intervals (positions)
     int32_t cnt[2];              // key tiles per interval walked by the CTA (union over both stages)
-    int32_t n_max;               // cnt[0] + cnt[1] (dual: the larger of the two stages' counts)
-    // Split-KV (decode) launches run "dual": both stages hold the same query rows and each takes its
-    // own key slice (interval st belongs to stage st), so a CTA keeps two slices in flight and one
-    // slice's softmax overlaps the other's MMAs.
-    int32_t dual;
-    int32_t q_st_stride;         // query-row distance between the stages (128, or 0 when dual)
-    int32_t out_st_stride;       // output-row distance between the stages (128, or rows per slice when dual)
+    int32_t n_max;               // the larger of the two stages' counts
+    int32_t out_st_stride;       // output-row distance between the stages' slices (rows per slice)
 };
 
 struct Shared {
@@ -88,7 +84,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
-attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+attn_split_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const AttnParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -100,9 +96,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.y, kvh = h / p.group;
 
-    // Thread 0 works out the CTA's geometry: heaviest (latest) causal tiles first; per stage the
-    // rows, positions and number of key tiles it takes part in.  Key tiles are walked interval 0
-    // first, then interval 1, in ascending position, so each stage's tiles are a prefix of the walk.
+    // Thread 0 works out the CTA's geometry: per stage the key slice and the number of key tiles.
     if (tid == 0) {
         Geom g;
         TileJob job;
@@ -110,35 +104,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         // An earlier CTA's wait expired: the launch is already lost, leave at once.
         if (p.status && *reinterpret_cast<volatile int32_t *>(p.status) != 0) g.found = 0;
         sh->abort_flag = 0;
-        g.dual = (p.splits > 1) ? 1 : 0;
-        g.q_st_stride = kTile;
-        g.out_st_stride = kTile;
-        if (g.found && !g.dual) {
-            g.q_row0 = (int32_t)job.q_row0; g.out_row0 = (int32_t)job.out_row0; g.kv_row0 = (int32_t)job.kv_row0;
-            g.cnt[0] = g.cnt[1] = 0;
-            for (int t = 0; t < 2; ++t) { g.lo[t] = (int32_t)job.iv_lo[t]; g.hi[t] = (int32_t)job.iv_hi[t]; }
-            for (int st = 0; st < 2; ++st) {
-                int32_t rows = job.n_rows - st * kTile;
-                rows = rows < 0 ? 0 : (rows > kTile ? kTile : rows);
-                g.rows[st] = rows;
-                g.pos0[st] = (int32_t)job.q_pos0 + st * kTile;
-                g.n[st] = 0;
-                if (rows > 0) {
-                    const int32_t last = g.pos0[st] + rows - 1;
-                    for (int t = 0; t < job.n_iv; ++t) {
-                        int32_t end = g.hi[t];
-                        if (p.causal && end > last + 1) end = last + 1;
-                        const int32_t c = end > g.lo[t] ? (end - g.lo[t] + kTile - 1) / kTile : 0;
-                        g.n[st] += c;
-                        g.cnt[t] = c > g.cnt[t] ? c : g.cnt[t];
-                    }
-                }
-            }
-            g.n_max = g.cnt[0] + g.cnt[1];
-        }
-        if (g.found && g.dual) {                              // stage st takes key slice 2 * blockIdx.z + st
+        if (g.found) {                                        // stage st takes key slice 2 * blockIdx.z + st (interval st)
             g.q_row0 = (int32_t)job.q_row0; g.kv_row0 = (int32_t)job.kv_row0;
-            g.q_st_stride = 0;
             g.out_st_stride = (int32_t)p.total_rows;
             g.out_row0 = (int32_t)job.out_row0 + 2 * (int32_t)blockIdx.z * (int32_t)p.total_rows;
             g.n_max = 0;
@@ -194,7 +161,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             mbar_arrive_expect_tx(bar_q, 2 * kTileBytes);
 #pragma unroll
             for (int st = 0; st < 2; ++st) {
-                const int row = sh->g.q_row0 + st * sh->g.q_st_stride;
+                const int row = sh->g.q_row0;                  // both stages hold the same rows
                 tma_load_3d(sQ + st * kTileBytes, &tm_q, bar_q, 0, h, row);
                 tma_load_3d(sQ + st * kTileBytes + kHalfTileBytes, &tm_q, bar_q, 64, h, row);
             }
@@ -210,13 +177,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 return true;
             };
             bool ok = true;
-            if (!sh->g.dual) {
-                for (int i = 0; i < 2 * n_max && ok; ++i) {    // items: K(0), V(0), K(1), V(1), ...
-                    const int jt = i >> 1, c0 = sh->g.cnt[0];
-                    const int krow = sh->g.kv_row0 + (jt < c0 ? sh->g.lo[0] + jt * kTile : sh->g.lo[1] + (jt - c0) * kTile);
-                    ok = load_tile((i & 1) ? (const void *)&tm_v : (const void *)&tm_k, krow);
-                }
-            } else {
+            {
                 // Each stage has its own key slice; items in the order the MMA issuer consumes them:
                 // K_0(0), K_1(0), then per step V_0(j), K_0(j+1), V_1(j), K_1(j+1).
                 const int n0 = sh->g.n[0], n1 = sh->g.n[1];
@@ -265,34 +226,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
             const int n_st[2] = {sh->g.n[0], sh->g.n[1]};
             bool ok = wait_bar(smem_u32(&sh->bar_q), 0, sh, p.status);
-            if (ok && !sh->g.dual) {
-                ok = kv_wait(0);
-                if (ok) {
-                    if (n_st[0] > 0) issue_qk(0, 0);
-                    if (n_st[1] > 0) issue_qk(1, 0);
-                    kv_release(0);
-                }
-                for (int j = 0; j < n_max && ok; ++j) {
-                    const bool has_next = j + 1 < n_max;
-                    ok = kv_wait(2 * j + 1);                   // V(j)
-#pragma unroll
-                    for (int st = 0; st < 2 && ok; ++st) {
-                        if (j < n_st[st]) {
-                            ok = wait_bar(smem_u32(&sh->p_ready[st]), j & 1, sh, p.status);
-                            if (!ok) break;
-                            tc_fence_after();
-                            issue_pv(st, 2 * j + 1, j > 0);
-                            if (j == n_st[st] - 1) tc_commit(smem_u32(&sh->o_final[st]));
-                        }
-                        if (st == 0 && has_next) { ok = kv_wait(2 * j + 2); if (!ok) break; }   // K(j+1)
-                        if (j + 1 < n_st[st]) issue_qk(st, 2 * j + 2);
-                    }
-                    if (!ok) break;
-                    kv_release(2 * j + 1);
-                    if (has_next) kv_release(2 * j + 2);
-                }
-            } else if (ok) {
-                // Dual: every ring item has one consumer; items arrive in the order used here.
+            if (ok) {
+                // Every ring item has one consumer; items arrive in the order used here.
                 int item = 0;
 #pragma unroll
                 for (int st = 0; st < 2 && ok; ++st) {
@@ -337,24 +272,17 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         const uint32_t tO = tmem + lane_base + kColO + st * kTile;
         const int n_mine = sh->g.n[st];
         const uint32_t bar_s = smem_u32(&sh->s_full[st]), bar_p = smem_u32(&sh->p_ready[st]);
-        // Per interval: where it ends, and the first key position that some row of this stage cannot
+        // Where the stage's slice ends, and the first key position that some row of this stage cannot
         // see (tiles reaching past it need the mask).
-        // (Dual launches: interval st is this stage's own key slice and the walk never changes interval.)
-        const bool dual = sh->g.dual != 0;
-        const int pos0 = sh->g.pos0[st], my_pos = pos0 + row_in_tile, cnt0 = dual ? 0x7fffffff : sh->g.cnt[0];
-        int iv_full[2], iv_mine[2];
-#pragma unroll
-        for (int t = 0; t < 2; ++t) {
-            const int hi_t = dual ? sh->g.hi[st] : sh->g.hi[t];
-            iv_full[t] = (p.causal && pos0 + 1 < hi_t) ? pos0 + 1 : hi_t;
-            iv_mine[t] = (p.causal && my_pos + 1 < hi_t) ? my_pos + 1 : hi_t;
-        }
-        int k0 = dual ? sh->g.lo[st] : sh->g.lo[0], cur = 0;
+        const int pos0 = sh->g.pos0[st], my_pos = pos0 + row_in_tile;
+        const int hi_st = sh->g.hi[st];
+        const int iv_full = (p.causal && pos0 + 1 < hi_st) ? pos0 + 1 : hi_st;
+        const int iv_mine = (p.causal && my_pos + 1 < hi_st) ? my_pos + 1 : hi_st;
+        int k0 = sh->g.lo[st];
 
         float m_ref = -INFINITY, l_run = 0.f;                // m_ref in log2 units of the scaled scores
         bool ok = true;
         for (int j = 0; j < n_mine; ++j, k0 += kTile) {
-            if (j == cnt0) { cur = 1; k0 = sh->g.lo[1]; }
             ok = __all_sync(0xffffffffu, wait_bar(bar_s, j & 1, sh, p.status));     // warp-uniform
             if (!ok) break;
             tc_fence_after();
@@ -362,9 +290,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             uint32_t r[kTile];
             tmem_ld128(tS, r);
             // Mask only when some row of this stage cannot see the whole tile.
-            const bool masked = k0 + kTile > (cur ? iv_full[1] : iv_full[0]);
+            const bool masked = k0 + kTile > iv_full;
             if (masked) {
-                int n_vis = (cur ? iv_mine[1] : iv_mine[0]) - k0;
+                int n_vis = iv_mine - k0;
                 n_vis = n_vis < 0 ? 0 : (n_vis > kTile ? kTile : n_vis);
 #pragma unroll
                 for (int c = 0; c < kTile; ++c) r[c] = (c < n_vis) ? r[c] : 0xff800000u;   // -inf
@@ -402,25 +330,15 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             float2 sum[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) sum[i] = make_float2(0.f, 0.f);
-            // p = 2^(s * scale - m): packed FMA for the argument, then the special-function unit, or for
-            // kPolyOf4 of every 4 pairs of an unmasked tile, the FMA/integer pipes.  P is packed to bf16
-            // pairs: column c of the A operand holds keys 2c (low half) and 2c+1 (high half).
-            if (masked) {
+            // p = 2^(s * scale - m): packed FMA for the argument, the special-function unit for 2^x, packed
+            // adds for the row sum.  P is packed to bf16 pairs: column c of the A operand holds keys 2c (low
+            // half) and 2c+1 (high half).
 #pragma unroll
-                for (int i = 0; i < kTile / 2; ++i) {
-                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, nm2);
-                    const float2 e = make_float2(ex2(x.x), ex2(x.y));
-                    sum[i & 3] = __fadd2_rn(sum[i & 3], e);
-                    r[i] = pack_bf16(e.x, e.y);
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < kTile / 2; ++i) {
-                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, nm2);
-                    const float2 e = ((i & 3) < kPolyOf4) ? ex2_poly2(x) : make_float2(ex2(x.x), ex2(x.y));
-                    sum[i & 3] = __fadd2_rn(sum[i & 3], e);
-                    r[i] = pack_bf16(e.x, e.y);
-                }
+            for (int i = 0; i < kTile / 2; ++i) {
+                const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, nm2);
+                const float2 e = make_float2(ex2(x.x), ex2(x.y));
+                sum[i & 3] = __fadd2_rn(sum[i & 3], e);
+                r[i] = pack_bf16(e.x, e.y);
             }
             const float2 s01 = __fadd2_rn(__fadd2_rn(sum[0], sum[1]), __fadd2_rn(sum[2], sum[3]));
             l_run += s01.x + s01.y;
@@ -511,50 +429,49 @@ static bool make_map(CUtensorMap *map, const void *base, int64_t rows, int32_t h
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int launch_attn_bf16(const AttnParams &p, cudaStream_t stream)
+}  // namespace splitk
+
+int launch_attn_split_bf16(const AttnParams &p, cudaStream_t stream)
 {
-    if (!p.status) { set_error("pec_prefill_attn: the bf16 path needs a status word"); return PEC_ERR_INVALID_ARG; }
+    using namespace splitk;
+    if (!p.status) { set_error("pec_decode_attn: the bf16 path needs a status word"); return PEC_ERR_INVALID_ARG; }
     // Rows the maps may touch: queries up to the chunk end, keys up to the end of the visible subset.
-    int64_t q_rows, kv_rows;
-    if (p.cu_seqlens) { q_rows = p.total_rows; kv_rows = p.total_rows; }
-    else {
-        q_rows = p.chunk_start + p.chunk_len;
-        kv_rows = 0;
-        for (int t = 0; t < p.n_iv; ++t) kv_rows = p.iv_hi[t] > kv_rows ? p.iv_hi[t] : kv_rows;
-    }
+    if (p.cu_seqlens) { set_error("pec_decode_attn: packed batches are not split"); return PEC_ERR_INVALID_ARG; }
+    const int64_t q_rows = p.chunk_start + p.chunk_len;
+    int64_t kv_rows = 0;
+    for (int t = 0; t < p.n_iv; ++t) kv_rows = p.iv_hi[t] > kv_rows ? p.iv_hi[t] : kv_rows;
     if (q_rows >= ((int64_t)1 << 31) || kv_rows >= ((int64_t)1 << 31)) {
-        set_error("pec_prefill_attn: more than 2^31 rows unsupported");
+        set_error("pec_decode_attn: more than 2^31 rows unsupported");
         return PEC_ERR_UNSUPPORTED;
     }
     CUtensorMap tm_q, tm_k, tm_v;
     if (!make_map(&tm_q, p.q, q_rows, p.Hq, p.q_stride_t, p.q_stride_h) ||
         !make_map(&tm_k, p.k, kv_rows, p.Hkv, p.k_stride_t, p.k_stride_h) ||
         !make_map(&tm_v, p.v, kv_rows, p.Hkv, p.v_stride_t, p.v_stride_h)) {
-        set_error("pec_prefill_attn: cuTensorMapEncodeTiled failed (driver too old, or strides/addresses not encodable)");
+        set_error("pec_decode_attn: cuTensorMapEncodeTiled failed (driver too old, or strides/addresses not encodable)");
         return PEC_ERR_CUDA;
     }
-    if (cudaFuncSetAttribute(attn_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) {
-        set_error("pec_prefill_attn: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
+    if (cudaFuncSetAttribute(attn_split_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) {
+        set_error("pec_decode_attn: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
         return PEC_ERR_CUDA;
     }
     // The softmax warpgroups take registers the third warpgroup gives up; that only works when the
     // launch allocation (registers per thread x threads) covers the new split.
     cudaFuncAttributes attr;
-    if (cudaFuncGetAttributes(&attr, attn_bf16_kernel) != cudaSuccess ||
+    if (cudaFuncGetAttributes(&attr, attn_split_bf16_kernel) != cudaSuccess ||
         attr.numRegs * kThreads < kSoftmaxWarps * 32 * kSoftmaxRegs + (kThreads - kSoftmaxWarps * 32) * kLightRegs) {
-        set_error("pec_prefill_attn: kernel register allocation too small for the warp-role register split");
+        set_error("pec_decode_attn: kernel register allocation too small for the warp-role register split");
         return PEC_ERR_CUDA;
     }
-    int64_t tiles = (p.total_rows + kBlockM - 1) / kBlockM;
-    if (p.cu_seqlens) tiles += p.B;
-    if (tiles > 0x7fffffff || p.Hq > 65535) { set_error("pec_prefill_attn: grid too large"); return PEC_ERR_UNSUPPORTED; }
-    if (p.splits < 1 || p.splits > 65535) { set_error("pec_prefill_attn: bad split count"); return PEC_ERR_INVALID_ARG; }
-    if (p.splits > 1 && p.total_rows > kTile) { set_error("pec_prefill_attn: split launches take at most 128 query rows"); return PEC_ERR_UNSUPPORTED; }
-    // Split launches are dual: each CTA's two stages take two consecutive key slices.
-    dim3 grid((unsigned)tiles, (unsigned)p.Hq, (unsigned)(p.splits > 1 ? (p.splits + 1) / 2 : 1));
-    attn_bf16_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, p);
+    const int64_t tiles = (p.total_rows + kBlockM - 1) / kBlockM;
+    if (tiles > 0x7fffffff || p.Hq > 65535) { set_error("pec_decode_attn: grid too large"); return PEC_ERR_UNSUPPORTED; }
+    if (p.splits < 1 || p.splits > 65535) { set_error("pec_decode_attn: bad split count"); return PEC_ERR_INVALID_ARG; }
+    if (p.total_rows > kTile) { set_error("pec_decode_attn: split launches take at most 128 query rows"); return PEC_ERR_UNSUPPORTED; }
+    // Each CTA's two stages take two consecutive key slices.
+    dim3 grid((unsigned)tiles, (unsigned)p.Hq, (unsigned)((p.splits + 1) / 2));
+    attn_split_bf16_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, p);
     const cudaError_t err = cudaGetLastError();
-    if (err != cudaSuccess) { set_error("pec_prefill_attn: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
+    if (err != cudaSuccess) { set_error("pec_decode_attn: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;
 }
 

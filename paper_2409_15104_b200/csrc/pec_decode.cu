@@ -124,7 +124,7 @@ static int run_decode(const pec_decode_args *a, const DecodeShape &shape, void *
     p.status = a->status;
     p.splits = shape.splits;
     p.split_keys = shape.split_keys;
-    const int rc = launch_attn_bf16(p, stream);
+    const int rc = launch_attn_split_bf16(p, stream);
     if (rc != PEC_OK) return rc;
     if (a->o_dtype == PEC_BF16)
         decode_reduce_kernel<true><<<a->Hq, kReduceThreads, 0, stream>>>(part_o, part_lse, a->o, a->lse, shape.splits, g, a->Hkv);

@@ -43,8 +43,8 @@ void zigzag_intervals(int64_t seq_len, int32_t num_parts, int32_t part_id, int32
 
 // Kernel launchers (each returns a pec_status).
 int launch_attn_f32(const AttnParams &p, cudaStream_t stream);
-int launch_attn_bf16(const AttnParams &p, cudaStream_t stream);
-int launch_attn_prefill_bf16(const AttnParams &p, cudaStream_t stream);
+int launch_attn_prefill_bf16(const AttnParams &p, cudaStream_t stream);   // every launch that is not split over the keys
+int launch_attn_split_bf16(const AttnParams &p, cudaStream_t stream);     // split-KV launches (decode)
 int launch_merge(const float *o_a, const float *lse_a, const float *o_b, const float *lse_b,
                  void *o_out, float *lse_out, int64_t items, int out_is_bf16, int inplace,
                  cudaStream_t stream);
