@@ -402,46 +402,56 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             uint8_t *my_row = stage_buf + lane * 256;
             const int sub = lane >> 4, chunk = lane & 15;                        // read-back: row parity and 16-byte chunk
             const int n_pass = p.o_is_bf16 ? 1 : 2;                              // 256 bytes of a row per pass
+            const int64_t row_bytes = (int64_t)p.Hq * kHeadDim * (p.o_is_bf16 ? 2 : 4);
+            uint8_t *out = static_cast<uint8_t *>(p.o) + (row0 + sub) * row_bytes + (int64_t)h * kHeadDim * (p.o_is_bf16 ? 2 : 4) + chunk * 16;
             for (int pass = 0; pass < n_pass; ++pass) {
+                if (p.o_is_bf16) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (!p.o_is_bf16 && (c >> 1) != pass) continue;
-                    uint32_t r[32];
-                    if (n_hf == 0) {
+                    for (int half = 0; half < 2; ++half) {                        // 64 channels = 8 chunks of 16 bytes
+                        uint32_t r[64];
+                        if (n_hf == 0) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = 0u;
-                    } else {
-                        tmem_ld32(tO + c * 32, r);
-                    }
-                    if (p.o_is_bf16) {
+                            for (int i = 0; i < 64; ++i) r[i] = 0u;
+                        } else {
+                            tmem_ld64(tO + half * 64, r);
+                        }
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {                             // 8 channels = 16 bytes per chunk
+                        for (int i = 0; i < 8; ++i) {
                             uint4 pk;
                             pk.x = pack_bf16(__uint_as_float(r[8 * i + 0]) * inv, __uint_as_float(r[8 * i + 1]) * inv);
                             pk.y = pack_bf16(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
                             pk.z = pack_bf16(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv);
                             pk.w = pack_bf16(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv);
-                            *reinterpret_cast<uint4 *>(my_row + (((c * 4 + i) ^ (lane & 15)) << 4)) = pk;
+                            *reinterpret_cast<uint4 *>(my_row + (((half * 8 + i) ^ (lane & 15)) << 4)) = pk;
                         }
-                    } else {
+                    }
+                } else {
+                    uint32_t r[64];                                               // 64 channels = 16 chunks of 16 bytes
+                    if (n_hf == 0) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {                             // 4 channels = 16 bytes per chunk
-                            const float4 f = make_float4(__uint_as_float(r[4 * i]) * inv, __uint_as_float(r[4 * i + 1]) * inv,
-                                                         __uint_as_float(r[4 * i + 2]) * inv, __uint_as_float(r[4 * i + 3]) * inv);
-                            *reinterpret_cast<float4 *>(my_row + ((((c & 1) * 8 + i) ^ (lane & 15)) << 4)) = f;
-                        }
+                        for (int i = 0; i < 64; ++i) r[i] = 0u;
+                    } else {
+                        tmem_ld64(tO + pass * 64, r);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float4 f = make_float4(__uint_as_float(r[4 * i]) * inv, __uint_as_float(r[4 * i + 1]) * inv,
+                                                     __uint_as_float(r[4 * i + 2]) * inv, __uint_as_float(r[4 * i + 3]) * inv);
+                        *reinterpret_cast<float4 *>(my_row + ((i ^ (lane & 15)) << 4)) = f;
                     }
                 }
                 __syncwarp();
-                uint8_t *out = static_cast<uint8_t *>(p.o) + (p.o_is_bf16 ? 0 : pass * 256) + chunk * 16;
-                const int64_t row_bytes = (int64_t)p.Hq * kHeadDim * (p.o_is_bf16 ? 2 : 4);
-                const int64_t head_bytes = (int64_t)h * kHeadDim * (p.o_is_bf16 ? 2 : 4);
-#pragma unroll 4
+                // All sixteen loads first, then the stores: two rows (2 x 256 contiguous bytes) per instruction.
+                uint4 val[16];
+#pragma unroll
                 for (int rr = 0; rr < 16; ++rr) {
                     const int row = 2 * rr + sub;
-                    const uint4 val = *reinterpret_cast<const uint4 *>(stage_buf + row * 256 + ((chunk ^ (row & 15)) << 4));
-                    if (row < rows_valid) *reinterpret_cast<uint4 *>(out + (row0 + row) * row_bytes + head_bytes) = val;
+                    val[rr] = *reinterpret_cast<const uint4 *>(stage_buf + row * 256 + ((chunk ^ (row & 15)) << 4));
                 }
+                uint8_t *dst = out + (p.o_is_bf16 ? 0 : pass * 256);
+#pragma unroll
+                for (int rr = 0; rr < 16; ++rr, dst += 2 * row_bytes)
+                    if (2 * rr + sub < rows_valid) *reinterpret_cast<uint4 *>(dst) = val[rr];
                 __syncwarp();
             }
             if (lane < rows_valid) p.lse[(row0 + lane) * p.Hq + h] = empty ? -INFINITY : m_ref * 0.6931471805599453f + logf(l_run);
