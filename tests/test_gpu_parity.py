@@ -161,6 +161,28 @@ def test_strided_inputs_and_custom_scale(pec, dtype):
     compare(o, lse, *want, *TOL[dtype], "strided")
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("shape", ["ramp", "spike", "falling"])
+def test_row_maximum_that_moves(pec, dtype, shape):
+    """Scores whose row maximum grows by far more than the lazy-rescale threshold (2^8) from one 64-key
+    half to the next ("ramp"), jumps once in the middle of the key range ("spike"), or only falls
+    ("falling": the accumulator is never rescaled).  Keys are multiples of one direction u, queries are u,
+    so score(key j) = c_j |u|^2 with c_j chosen per shape; V stays random."""
+    S, hq, hkv = 700, 2, 1
+    q, k, v = _qkv(7100, S, hq, hkv, dtype)
+    u = workloads.normal_tensor(7101, 1, (128,), torch.float32)
+    u = u / u.norm() * (128 ** 0.25)                     # |u|^2 * scale = 1
+    j = torch.arange(S, dtype=torch.float32)
+    c = {"ramp": j * 0.2, "spike": torch.where(j == 333, torch.tensor(60.0), torch.tensor(0.0)) + 0.01 * torch.sin(j),
+         "falling": (S - j) * 0.2}[shape]
+    k = (c[:, None, None] * u[None, None, :]).expand(S, hkv, 128).to(dtype).contiguous()
+    q = (u[None, None, :] * torch.ones(S, hq, 1)).to(dtype).contiguous()
+    want = oracle.prefill_attn(q, k, v, seq_len=S)
+    o, lse = pec.pec_prefill_attn(*_gpu(q, k, v))
+    pec.check_status()
+    compare(o, lse, *want, *TOL[dtype], f"moving maximum {shape} {dtype}")
+
+
 # ------------------------------------------------------------------ packed batches
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
 @pytest.mark.parametrize("lens", [[5], [128, 128], [1, 300, 0, 77, 129, 64], [200, 1, 1, 511]])
