@@ -28,6 +28,10 @@ from paper_2409_15104_b200 import workloads
 METRIC = "causal prefill attention TFLOP/s (tokens/s and % of dense BF16 peak alongside), 1 B200"
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes (read + write) of one attention launch, from the ncu capture summarised in
+# profiles/attn_prefill_bf16_kernel_c3.md (mean of its two launches).  Valid for that kernel and workload
+# only: set an entry back to None when the kernel changes.
+NCU_TRAFFIC_BYTES = {"c3": 767.3e6}
 
 
 def load_peaks():
@@ -292,7 +296,8 @@ def run_ours(args, wl):
         "merge": merge,
         "roofline": {"bound": "tensor", "kernel": "attn_prefill_bf16_kernel", "achieved": attn_tflops,
                      "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": attn_tflops / peaks["bf16_sustained"],
-                     "traffic": None, "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step)",
+                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "traffic_unit": "bytes per launch (ncu dram read + write)",
+                     "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step)",
                      "frac_of_burst": attn_tflops / peaks["bf16_burst"], "frac_of_nominal": attn_tflops / NOMINAL_BF16_TFLOPS,
                      "flops_per_launch": flops_launch, "ms_per_launch": attn_avg_ms},
         "cpu_baseline": {"value": cpu["tflops"], "unit": "TFLOP/s", "cores": cpu["cores"], "kind": "oracle",
