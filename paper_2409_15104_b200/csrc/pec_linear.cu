@@ -55,7 +55,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 2)
 linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-                   __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t *status)
+                   __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t band, int32_t *status)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -63,8 +63,17 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
     Shared *sh = reinterpret_cast<Shared *>(smem_raw + (ring - raw) + kSlots * kSlotBytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_ctarank();                  // 0 = leader
-    const int64_t m0 = (int64_t)(blockIdx.x >> 1) * (2 * kBM) + rank * kBM;
-    const int n0 = blockIdx.y * kBN;
+    // Tile order.  Clusters are dispatched x-fastest; taken as they come (all row pairs of one column
+    // of y, then the next column) every column would stream the whole of x from HBM again.  The
+    // dispatch index is re-read as bands of `band` row pairs: within a band the row pairs vary fastest
+    // and the columns next, so a band's rows of x (and all of w) stay in L2 while its columns are done.
+    const int pairs = (int)(gridDim.x >> 1), gn = (int)gridDim.y;
+    const int64_t seq = (int64_t)blockIdx.y * pairs + (blockIdx.x >> 1);
+    const int band_i = (int)(seq / ((int64_t)band * gn));
+    const int band_pairs = (pairs - band_i * band) < band ? (pairs - band_i * band) : band;
+    const int within = (int)(seq - (int64_t)band_i * band * gn);
+    const int64_t m0 = (int64_t)(band_i * band + within % band_pairs) * (2 * kBM) + rank * kBM;
+    const int n0 = (within / band_pairs) * kBN;
     const int n_kb = (K + kBK - 1) / kBK;
 
     if (tid == 0) {
@@ -210,9 +219,13 @@ extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_
     }
     const int64_t pairs = (M + 2 * lin::kBM - 1) / (2 * lin::kBM), gn = (N + lin::kBN - 1) / lin::kBN;
     if (gn > 65535) { set_error("pec_linear: N too large"); return PEC_ERR_UNSUPPORTED; }
+    // Rows of x per band: what leaves room for w in about 96 MB of the L2 (at least 4 row pairs, at most 32).
+    const int64_t w_bytes = (int64_t)N * K * 2, pair_bytes = (int64_t)2 * lin::kBM * K * 2;
+    int64_t band = ((int64_t)96 << 20) > w_bytes ? (((int64_t)96 << 20) - w_bytes) / pair_bytes : 0;
+    band = band < 4 ? 4 : (band > 32 ? 32 : band);
     dim3 grid((unsigned)(2 * pairs), (unsigned)gn);           // clusters of two CTAs along x
     lin::linear_kernel<<<grid, lin::kThreads, lin::kSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(
-        tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, status);
+        tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, (int32_t)band, status);
     const cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("pec_linear: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;
