@@ -10,19 +10,20 @@
 //   warp  9     TMA loader (Q once, then K and V tiles through a ring of shared-memory slots)
 //   warp  11    idle; it completes the third warpgroup so that it can hand its registers to the
 //               softmax warpgroups (setmaxnreg acts on whole warpgroups)
-// K and V arrive as 128-key tiles, but scores are produced and consumed in halves of 64 keys: each
-// stage owns two 64-column score buffers in tensor memory, and half h uses buffer h & 1.
-// S(h) = Q K_h^T lands in its buffer, the softmax warps turn it into P(h) (bf16, written over the
-// first 32 columns of the same buffer), and O += P(h) V_h accumulates in tensor memory.  S(h+1)
-// sits in the other buffer, so it is issued before the softmax of half h is done; per stage the
-// issue order is
-//   PV(h), S(h+2), PV(h+1), S(h+3), ...
-// interleaved between the two stages: a stage's softmax finds its next scores waiting, and the
-// tensor pipe has the other buffer's and the other stage's work queued.  The accumulator is
-// rescaled lazily: the reference maximum of a row only moves when the new maximum exceeds it by
-// 2^8, and a warp that has to rescale first waits for the PV product still in flight on its O.
+// K and V arrive as 128-key tiles and a tile's scores are one 128 x 128 product (N = 128 halves the
+// shared-memory traffic of the Q operand per FLOP against 64-key products, and shared-memory
+// bandwidth is what the tensor pipe waits for here).  Tensor memory has room for one such score
+// buffer beside the two accumulators, so BOTH stages share it, in turns: S_0(j) lands in it, the
+// softmax warps of stage 0 pull their rows into registers (128 per thread) and hand the buffer back
+// at once; S_1(j) follows while stage 0 is still at its exponentials, then S_0(j+1), and so on.
+// P (bf16) goes to a region of its own per stage, so a product O += P(j) V_j never holds the score
+// buffer.  Per stage the issue order is S(j+1), PV(j): the next scores wait in the buffer (or are on
+// their way) when the stage's softmax comes back for them, and the tensor pipe always has the other
+// stage's work queued.  The accumulator is rescaled lazily: the reference maximum of a row only moves
+// when the new maximum exceeds it by 2^8, and a warp that has to rescale first waits for the PV
+// product still in flight on its O.
 //
-// TMEM columns: stage s scores [128 s, 128 s + 128) as two buffers of 64; O_s [256 + 128 s, +128).
+// TMEM columns: scores [0, 128); P_s [128 + 64 s, +64); O_s [256 + 128 s, +128).
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -35,7 +36,7 @@ using namespace sm100;
 namespace pf {
 
 constexpr int kTile = 128;                                 // rows per stage, keys per K/V tile
-constexpr int kHalf = 64;                                  // keys per score buffer
+constexpr int kHalf = 64;                                  // keys per call of the four-step PV helper
 constexpr int kBlockM = 2 * kTile;                         // query rows per CTA
 constexpr int kStages = 4;                                 // K/V ring slots
 constexpr int kThreads = 384;                              // three full warpgroups
@@ -45,7 +46,7 @@ constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;          // one TMA box: 128 r
 constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;        // 128 x 128 bf16
 constexpr uint32_t kKeyHalfBytes = kHalf * 128;            // 64 rows of a box (128 bytes per row)
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256;                 // + 128 * stage
+constexpr uint32_t kColS = 0, kColP = 128, kColO = 256;    // P: + 64 * stage; O: + 128 * stage
 constexpr float kRescaleThreshold = 8.0f;                  // log2 units
 constexpr long long kWaitCycles = 2000000000LL;            // bounded waits give up after ~1 s
 constexpr uint32_t kSuspendNs = 2000;                      // a waiting thread sleeps in the barrier unit this long per try
@@ -66,7 +67,7 @@ struct Geom {
 struct Shared {
     uint64_t bar_q;
     uint64_t kv_full[kStages], kv_empty[kStages];
-    uint64_t s_full[2][2], p_ready[2][2];   // [stage][buffer]
+    uint64_t s_full[2], s_taken[2], p_ready[2];   // [stage], one phase per key tile
     uint64_t pv_done[2];                     // one phase per PV product of the stage
     uint64_t o_final[2];                     // the stage's last PV product is done
     Geom g;
@@ -143,10 +144,9 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         mbar_init(smem_u32(&sh->bar_q), 1);
         for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->kv_full[s]), 1); mbar_init(smem_u32(&sh->kv_empty[s]), 2); }
         for (int st = 0; st < 2; ++st) {
-            for (int b = 0; b < 2; ++b) {
-                mbar_init(smem_u32(&sh->s_full[st][b]), 1);
-                mbar_init(smem_u32(&sh->p_ready[st][b]), 4);  // one arrival per softmax warp
-            }
+            mbar_init(smem_u32(&sh->s_full[st]), 1);
+            mbar_init(smem_u32(&sh->s_taken[st]), 4);         // one arrival per softmax warp
+            mbar_init(smem_u32(&sh->p_ready[st]), 4);
             mbar_init(smem_u32(&sh->pv_done[st]), 1);
             mbar_init(smem_u32(&sh->o_final[st]), 1);
         }
@@ -193,71 +193,89 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         // The whole warp walks the loop and one elected lane issues: addresses, descriptors and loop
         // state stay warp-uniform, which keeps the instruction count per MMA low.  An issuer shares its
         // scheduler with two softmax warps, and one warp issuing for both stages was the kernel's
-        // bottleneck; the two stages touch disjoint tensor memory, so their MMAs need no order between
-        // them.  Each issuer waits for and releases every ring item, used by its stage or not, so the
-        // "empty" barriers always see two arrivals per item.
+        // bottleneck.  The stages' accumulators and P regions are disjoint; the score buffer they share is
+        // handed from one to the other through the "taken" barriers.  Each issuer waits for and releases
+        // every ring item, used by its stage or not, so the "empty" barriers always see two arrivals per item.
         reg_dealloc<kLightRegs>();
         if (n_max > 0) {
             const int st = (warp == kMmaWarp0) ? 0 : 1;
             const bool leader = elect_one();
-            constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kHalf, 0, 0);
+            constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kTile, 0, 0);
             constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, kHeadDim, 0, 1);
             auto wait_u = [&](uint64_t *bar, uint32_t parity) {
                 return __all_sync(0xffffffffu, wait_bar(smem_u32(bar), parity, sh, p.status));
             };
             auto kv_wait = [&](int item) { return wait_u(&sh->kv_full[item % kStages], (item / kStages) & 1); };
             auto kv_release = [&](int item) { if (leader) tc_commit(smem_u32(&sh->kv_empty[item % kStages])); };
-            const uint32_t tS = tmem + kColS + st * kTile, tO = tmem + kColO + st * kTile;
+            const uint32_t tS = tmem + kColS, tP = tmem + kColP + st * 64, tO = tmem + kColO + st * kTile;
             // Descriptors: the stage's Q tile gives eight fixed A descriptors (16 channels per K step, four steps
-            // per 64-channel box); a K or V half is the ring's first descriptor plus slot and half offsets.
+            // per 64-channel box); a K or V tile is the ring's first descriptor plus the slot offset.
             constexpr uint32_t kBox16 = kHalfTileBytes >> 4;
             uint64_t a_desc[8];
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
                 a_desc[ks] = smem_desc_sw128(sQ + st * kTileBytes + (uint32_t)(ks >> 2) * kHalfTileBytes + (uint32_t)(ks & 3) * 32u, 16, 1024);
             const uint64_t k_ring = smem_desc_sw128(sRing, 16, 1024), v_ring = smem_desc_sw128(sRing, kHalfTileBytes, 1024);
-            // S(hf) = Q K^T for the 64 keys of half hf (tile hf / 2, rows 64 (hf & 1) .. of it): both operands
-            // K-major; the half's rows start 8 KiB into each box.
-            auto issue_qk = [&](int hf) {
-                const int item = 2 * (hf >> 1), b = hf & 1;
-                const uint64_t k0 = k_ring + (uint32_t)(((item % kStages) * kTileBytes + b * kKeyHalfBytes) >> 4);
-                if (leader) mma_ss_k128_commit<kBox16>(tS + b * kHalf, a_desc, k0, idesc_qk, smem_u32(&sh->s_full[st][b]));
+            const int n_st = sh->g.n[st], n_ot = sh->g.n[st ^ 1];
+            // S(j) = Q K_j^T for the 128 keys of tile j, both operands K-major, into the shared score buffer.
+            auto issue_qk = [&](int j) {
+                const uint64_t k0 = k_ring + (uint32_t)((((2 * j) % kStages) * kTileBytes) >> 4);
+                if (leader) mma_ss_k128_commit<kBox16>(tS, a_desc, k0, idesc_qk, smem_u32(&sh->s_full[st]));
             };
-            // O (+)= P(hf) V: A = P from TMEM (8 columns per 16 keys), B = the half's 64 keys of the V tile
-            // stored [key][channel] (N-contiguous): 16 keys = 2048 bytes per step, channel halves 16 KiB apart.
-            auto issue_pv = [&](int hf, bool last) {
-                const int item = 2 * (hf >> 1) + 1, b = hf & 1;
-                const uint64_t v0 = v_ring + (uint32_t)(((item % kStages) * kTileBytes + b * kKeyHalfBytes) >> 4);
+            // O (+)= P(j) V_j: A = P from TMEM (8 columns per 16 keys), B = the V tile stored [key][channel]
+            // (N-contiguous): 16 keys = 2048 bytes per step, channel halves 16 KiB apart.
+            auto issue_pv = [&](int j, bool last) {
+                const uint64_t v0 = v_ring + (uint32_t)((((2 * j + 1) % kStages) * kTileBytes) >> 4);
                 if (leader) {
-                    mma_ts_k64(tO, tS + b * kHalf, v0, idesc_pv, hf > 0 ? 1u : 0u);
+                    mma_ts_k64(tO, tP, v0, idesc_pv, j > 0 ? 1u : 0u);
+                    mma_ts_k64(tO, tP + 32, v0 + (kKeyHalfBytes >> 4), idesc_pv, 1u);
                     tc_commit(smem_u32(&sh->pv_done[st]));
                     if (last) tc_commit(smem_u32(&sh->o_final[st]));
                 }
             };
+            // The score buffer is used in the order (0,0), (1,0), (0,1), (1,1), ... (stage, tile), a stage that has
+            // run out of tiles dropping out; S(j) may be issued once the previous user's softmax warps hold
+            // their scores in registers.
+            auto wait_buffer = [&](int j) {
+                int pst, pj;
+                if (st == 0) {
+                    if (j == 0) return true;
+                    pst = (j - 1 < n_ot) ? 1 : 0; pj = j - 1;
+                } else {
+                    if (j < n_ot) { pst = 0; pj = j; }
+                    else if (j > 0) { pst = 1; pj = j - 1; }
+                    else return true;
+                }
+                const bool got = wait_u(&sh->s_taken[pst], pj & 1);
+                if (got) tc_fence_after();
+                return got;
+            };
 
-            const int n_hf = 2 * sh->g.n[st];                  // halves of this stage
             bool ok = wait_u(&sh->bar_q, 0) && kv_wait(0);
             if (ok) {
-                if (n_hf > 0) { issue_qk(0); issue_qk(1); }
+                if (n_st > 0) { ok = wait_buffer(0); if (ok) issue_qk(0); }
                 kv_release(0);
             }
-            for (int hf = 0; hf < 2 * n_max && ok; ++hf) {
-                const int j = hf >> 1, b = hf & 1;
-                const bool has_next = j + 1 < n_max;
-                if (b == 0) ok = kv_wait(2 * j + 1);           // V(j)
-                if (ok && hf < n_hf) {
-                    ok = wait_u(&sh->p_ready[st][b], j & 1);
+            for (int j = 0; j < n_max && ok; ++j) {
+                if (j + 1 < n_max) {
+                    ok = kv_wait(2 * j + 2);                       // K(j+1)
+                    if (!ok) break;
+                    if (j + 1 < n_st) {
+                        ok = wait_buffer(j + 1);
+                        if (!ok) break;
+                        issue_qk(j + 1);
+                    }
+                    kv_release(2 * j + 2);
+                }
+                ok = kv_wait(2 * j + 1);                           // V(j)
+                if (!ok) break;
+                if (j < n_st) {
+                    ok = wait_u(&sh->p_ready[st], j & 1);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(hf, hf == n_hf - 1);
+                    issue_pv(j, j == n_st - 1);
                 }
-                if (ok && b == 0 && has_next) ok = kv_wait(2 * j + 2);   // K(j+1)
-                if (!ok) break;
-                if (hf + 2 < n_hf) issue_qk(hf + 2);
-                if (b == 1) {
-                    kv_release(2 * j + 1);
-                    if (has_next) kv_release(2 * j + 2);
-                }
+                kv_release(2 * j + 1);
             }
         }
         __syncwarp();
@@ -273,13 +291,14 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         const int st = warp >> 2, quarter = warp & 3;
         const int row_in_tile = quarter * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-        const uint32_t tS = tmem + lane_base + kColS + st * kTile;
+        const uint32_t tS = tmem + lane_base + kColS;
+        const uint32_t tP = tmem + lane_base + kColP + st * 64;
         const uint32_t tO = tmem + lane_base + kColO + st * kTile;
-        const int n_hf = 2 * sh->g.n[st];
+        const int n_t = sh->g.n[st], n_hf = 2 * n_t;
         const uint32_t bar_pv = smem_u32(&sh->pv_done[st]);
         // Per interval: where it ends, and the first key position that some row of this stage cannot
-        // see (halves reaching past it need the mask).
-        const int pos0 = sh->g.pos0[st], my_pos = pos0 + row_in_tile, hf0 = 2 * sh->g.cnt[0];
+        // see (tiles reaching past it need the mask).
+        const int pos0 = sh->g.pos0[st], my_pos = pos0 + row_in_tile, t0 = sh->g.cnt[0];
         int iv_full[2], iv_mine[2];
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
@@ -291,97 +310,89 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 
         float m_ref = -INFINITY, l_run = 0.f;                // m_ref in log2 units of the scaled scores
         bool ok = true;
-        // The special-function unit is the softmax's bottleneck and this warp shares its scheduler's
-        // unit with the warp of the other stage that has the same quarter.  The two take turns at the
-        // exponentials of a half (a token passed through two named barriers), so one warp's loads,
-        // maxima and stores run under the other's exponentials instead of both phases colliding.
-        // The turns cover the halves both stages have; a warp whose wait failed keeps passing the
-        // token (and does nothing else) so that its partner never blocks on it.
-        const int n_turns = 2 * (sh->g.n[0] < sh->g.n[1] ? sh->g.n[0] : sh->g.n[1]);
-        const uint32_t tok_mine = 1 + 2 * quarter + st, tok_other = 1 + 2 * quarter + (st ^ 1);
-        if (st == 1 && n_turns > 0) named_arrive64(tok_other);   // stage 0 goes first
-        for (int hf = 0; hf < n_hf; ++hf, k0 += kHalf) {
-            if (hf == hf0) { cur = 1; k0 = sh->g.lo[1]; }
-            const int b = hf & 1;
-            const bool turn = hf < n_turns;
-            uint32_t r[kHalf];
-            float2 sc2, nm2;
-            if (ok) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->s_full[st][b]), (hf >> 1) & 1, sh, p.status));   // warp-uniform
-            if (ok) {
-                tc_fence_after();
-                tmem_ld64(tS + b * kHalf, r);
-                // Mask only when some row of this stage cannot see the whole half.
-                const bool masked = k0 + kHalf > (cur ? iv_full[1] : iv_full[0]);
-                if (masked) {
-                    int n_vis = (cur ? iv_mine[1] : iv_mine[0]) - k0;
-                    n_vis = n_vis < 0 ? 0 : (n_vis > kHalf ? kHalf : n_vis);
+        for (int j = 0; j < n_t && ok; ++j, k0 += kTile) {
+            if (j == t0) { cur = 1; k0 = sh->g.lo[1]; }
+            uint32_t r[kTile];
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->s_full[st]), j & 1, sh, p.status));   // warp-uniform
+            if (!ok) break;
+            tc_fence_after();
+            tmem_ld128(tS, r);
+            // The scores are in registers: the buffer may take the other stage's next tile.
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->s_taken[st]));
+            // Mask only when some row of this stage cannot see the whole tile.
+            const bool masked = k0 + kTile > (cur ? iv_full[1] : iv_full[0]);
+            if (masked) {
+                int n_vis = (cur ? iv_mine[1] : iv_mine[0]) - k0;
+                n_vis = n_vis < 0 ? 0 : (n_vis > kTile ? kTile : n_vis);
 #pragma unroll
-                    for (int c = 0; c < kHalf; ++c) r[c] = (c < n_vis) ? r[c] : 0xff800000u;   // -inf
-                }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                for (int c = 0; c < kTile; ++c) r[c] = (c < n_vis) ? r[c] : 0xff800000u;   // -inf
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < kHalf; c += 8) {
-                    mx0 = fmax3(mx0, __uint_as_float(r[c + 0]), __uint_as_float(r[c + 1]));
-                    mx1 = fmax3(mx1, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
-                    mx2 = fmax3(mx2, __uint_as_float(r[c + 4]), __uint_as_float(r[c + 5]));
-                    mx3 = fmax3(mx3, __uint_as_float(r[c + 6]), __uint_as_float(r[c + 7]));
-                }
-                const float m_new = fmax3(mx0, mx1, fmaxf(mx2, mx3)) * p.scale_log2;   // -inf stays -inf (scale > 0)
+            for (int c = 0; c < kTile; c += 8) {
+                mx0 = fmax3(mx0, __uint_as_float(r[c + 0]), __uint_as_float(r[c + 1]));
+                mx1 = fmax3(mx1, __uint_as_float(r[c + 2]), __uint_as_float(r[c + 3]));
+                mx2 = fmax3(mx2, __uint_as_float(r[c + 4]), __uint_as_float(r[c + 5]));
+                mx3 = fmax3(mx3, __uint_as_float(r[c + 6]), __uint_as_float(r[c + 7]));
+            }
+            const float m_new = fmax3(mx0, mx1, fmaxf(mx2, mx3)) * p.scale_log2;   // -inf stays -inf (scale > 0)
 
-                // Lazy rescale: move the reference maximum only when it is outgrown by 2^8.
-                float alpha = 1.f;
-                const bool grow = m_new > m_ref + kRescaleThreshold;
-                if (grow) {
-                    alpha = ex2(m_ref - m_new);                   // 0 when the row had no key so far
-                    m_ref = m_new;
-                    l_run *= alpha;
-                }
-                if (hf > 0 && __any_sync(0xffffffffu, grow)) {
-                    // O still receives P(hf-1) V: wait for that product (phase hf-1 of the stage's PV barrier;
-                    // PV(hf) cannot be issued before this warp hands P(hf) over, so the phase is unambiguous).
-                    ok = __all_sync(0xffffffffu, wait_bar(bar_pv, (hf - 1) & 1, sh, p.status));
-                    if (ok) {
-                        tc_fence_after();
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t o[32];
-                            tmem_ld32(tO + c * 32, o);
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                            tmem_st32(tO + c * 32, o);
-                        }
-                    }
-                }
-                const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-                sc2 = make_float2(p.scale_log2, p.scale_log2);
-                nm2 = make_float2(neg_m, neg_m);
+            // Lazy rescale: move the reference maximum only when it is outgrown by 2^8.
+            float alpha = 1.f;
+            const bool grow = m_new > m_ref + kRescaleThreshold;
+            if (grow) {
+                alpha = ex2(m_ref - m_new);                   // 0 when the row had no key so far
+                m_ref = m_new;
+                l_run *= alpha;
             }
-            if (turn) named_sync64(tok_mine);
-            if (ok) {
-                float2 sum[4];
+            bool pv_waited = (j == 0);
+            if (j > 0 && __any_sync(0xffffffffu, grow)) {
+                // O still receives P(j-1) V: wait for that product (phase j-1 of the stage's PV barrier; PV(j)
+                // cannot be issued before this warp hands P(j) over, so the phase is unambiguous).
+                ok = __all_sync(0xffffffffu, wait_bar(bar_pv, (j - 1) & 1, sh, p.status));
+                if (!ok) break;
+                pv_waited = true;
+                tc_fence_after();
 #pragma unroll
-                for (int i = 0; i < 4; ++i) sum[i] = make_float2(0.f, 0.f);
-                // p = 2^(s * scale - m): packed FMA for the argument, the special-function unit for 2^x, packed
-                // adds for the row sum.  P is packed to bf16 pairs: column c of the A operand holds keys 2c (low
-                // half) and 2c+1 (high half); r[i] is reused for pair i.
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
 #pragma unroll
-                for (int i = 0; i < kHalf / 2; ++i) {
-                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, nm2);
-                    const float2 e = make_float2(ex2(x.x), ex2(x.y));
-                    sum[i & 3] = __fadd2_rn(sum[i & 3], e);
-                    r[i] = pack_bf16(e.x, e.y);
+                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    tmem_st32(tO + c * 32, o);
                 }
-                const float2 s01 = __fadd2_rn(__fadd2_rn(sum[0], sum[1]), __fadd2_rn(sum[2], sum[3]));
-                l_run += s01.x + s01.y;
             }
-            if (turn && !(st == 1 && hf == n_turns - 1)) named_arrive64(tok_other);
-            if (ok) {
-                tmem_st32(tS + b * kHalf, r);
-                tmem_st_wait();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sh->p_ready[st][b]));
+            const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+            const float2 sc2 = make_float2(p.scale_log2, p.scale_log2), nm2 = make_float2(neg_m, neg_m);
+            float2 sum[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) sum[i] = make_float2(0.f, 0.f);
+            // p = 2^(s * scale - m): packed FMA for the argument, the special-function unit for 2^x, packed
+            // adds for the row sum.  P is packed to bf16 pairs: column c of the A operand holds keys 2c (low
+            // half) and 2c+1 (high half); r[i] is reused for pair i.
+#pragma unroll
+            for (int i = 0; i < kTile / 2; ++i) {
+                const float2 x = __ffma2_rn(make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1])), sc2, nm2);
+                const float2 e = make_float2(ex2(x.x), ex2(x.y));
+                sum[i & 3] = __fadd2_rn(sum[i & 3], e);
+                r[i] = pack_bf16(e.x, e.y);
             }
+            const float2 s01 = __fadd2_rn(__fadd2_rn(sum[0], sum[1]), __fadd2_rn(sum[2], sum[3]));
+            l_run += s01.x + s01.y;
+            // P(j-1) is read by its product until that is done.
+            if (!pv_waited) {
+                ok = __all_sync(0xffffffffu, wait_bar(bar_pv, (j - 1) & 1, sh, p.status));
+                if (!ok) break;
+                tc_fence_after();
+            }
+            tmem_st32(tP, r);
+            tmem_st32(tP + 32, r + 32);
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->p_ready[st]));
         }
 
         // Epilogue: O / l and LSE = ln2 * m + ln l; rows without any visible key give 0 and -inf.
