@@ -252,6 +252,40 @@ int pec_plan_partitions(int64_t seq_len, int32_t num_parts, int64_t chunk_len, i
                         int32_t block_m, int32_t block_n, int32_t causal, pec_plan *plan);
 
 /*
+ * Work plan of ring-attention sequence parallelism over num_parts ranks (Section 2.2: each replica
+ * keeps the queries of its own segment and the K/V segments travel round the ring, one hop per
+ * step).  Rank r owns the query rows of its segment; at ring step t it holds the K/V segment of
+ * rank (r - t) mod num_parts.  pairs[r * num_parts + t] = number of visible (query, key) pairs of
+ * that rank at that step: the attention work of the step (x 4 * D * Hq FLOPs).  step_max[t] = the
+ * largest entry of step t over the ranks (a ring step lasts as long as its slowest rank),
+ * rank_total[r] = the row sum of rank r.
+ * layout PEC_LAYOUT_ZIGZAG: segment r = zigzag partition r of pec_plan_partitions (blocks r and
+ * 2P-1-r).  layout PEC_LAYOUT_CONTIGUOUS: segment r = [c[r], c[r+1]) with
+ * c[k] = min(seq_len, align * floor(k * U / P)), U = ceil(seq_len / align): the split that leaves
+ * the last rank with about 2P-1 times the causal work of the first, which the zigzag pairing
+ * removes (there every off-diagonal step costs the same on every rank).  The paper names neither
+ * rule; both are this library's.
+ * All arrays are host memory owned by the caller and may be NULL to skip; pairs_cap >= P*P,
+ * vec_cap >= P where given.  Errors: INVALID_ARG (sizes, unknown layout), CAPACITY.
+ */
+typedef enum { PEC_LAYOUT_ZIGZAG = 0, PEC_LAYOUT_CONTIGUOUS = 1 } pec_layout;
+int pec_plan_ring(int64_t seq_len, int32_t num_parts, int32_t align, int32_t layout, int32_t causal,
+                  int64_t *pairs, int64_t pairs_cap, int64_t *step_max, int64_t *rank_total, int64_t vec_cap);
+
+/*
+ * Token-balanced short-request batches (Section 5.2: when short prefills preempt a long one, the
+ * batches are built so that the total number of tokens per batch is balanced across the model
+ * replicas).  The paper states the goal, not the rule; this library's rule is longest-first
+ * greedy: requests are taken in order of decreasing length (equal lengths: lower index first) and
+ * each goes to the replica that has the fewest tokens so far (equal totals: lowest replica id).
+ * The largest replica total is then at most 4/3 - 1/(3 R) times the best possible one.
+ * lengths: host [n], each >= 0; assign: host [n], receives the replica id of every request;
+ * tokens: host [replicas] or NULL, receives the token total of every replica.
+ * Errors: INVALID_ARG (NULL lengths/assign with n > 0, n < 0, replicas < 1, a negative length).
+ */
+int pec_balance_batches(const int32_t *lengths, int32_t n, int32_t replicas, int32_t *assign, int64_t *tokens);
+
+/*
  * Intra-node SP strategy selection for a long prefill (Section 5.3).  With TP size T, G GPUs per
  * node, per-GPU segment length s, model width d, N_h query heads and N_kv KV heads of size d_h, the
  * paper gives, per stage and strategy, the communication volume in a node and the computation

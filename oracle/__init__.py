@@ -13,6 +13,9 @@ from .reference import (  # noqa: F401
     select_sp,
     linear,
     plan_partitions,
+    plan_ring,
+    ring_segments,
+    balance_batches,
     partition_intervals,
     oracle_threads,
     SKIP,

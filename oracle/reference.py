@@ -242,6 +242,68 @@ def merge_n(o_parts, lse_parts):
 
 
 # --------------------------------------------------------------------------- SP strategy cost model
+def ring_segments(seq_len, num_parts, align, layout):
+    """Row intervals of every ring rank's segment: layout "zigzag" pairs block r with block 2P-1-r of
+    2P equal blocks, layout "contiguous" cuts P blocks; block bounds are align * floor(k*U/nblocks)
+    with U = ceil(S/align), cut at S."""
+    S, P = int(seq_len), int(num_parts)
+    U = _ceil_div(S, align)
+    if layout == "zigzag":
+        b = [min(S, align * ((k * U) // (2 * P))) for k in range(2 * P + 1)]
+        return [[(b[r], b[r + 1]), (b[2 * P - 1 - r], b[2 * P - r])] for r in range(P)]
+    if layout == "contiguous":
+        b = [min(S, align * ((k * U) // P)) for k in range(P + 1)]
+        return [[(b[r], b[r + 1])] for r in range(P)]
+    raise ValueError("unknown layout")
+
+
+def plan_ring(seq_len, num_parts, align, layout, causal):
+    """Work of ring-attention sequence parallelism (Section 2.2), counted row by row.
+
+    Rank r keeps the query rows of its segment; at step t it holds the keys of the segment of rank
+    (r - t) mod P.  pairs[r][t] = sum over the rank's rows i of the number of those keys visible to
+    row i (keys j <= i under the causal mask, else all of them).  step_max[t] = max over ranks,
+    rank_total[r] = sum over steps.
+    """
+    S, P = int(seq_len), int(num_parts)
+    if S < 0 or P < 1 or align < 1:
+        raise ValueError("bad planner arguments")
+    seg = ring_segments(S, P, align, layout)
+    pairs = [[0] * P for _ in range(P)]
+    for r in range(P):
+        for t in range(P):
+            keys = seg[(r - t) % P]
+            n = 0
+            for q_lo, q_hi in seg[r]:
+                for i in range(q_lo, q_hi):
+                    for k_lo, k_hi in keys:
+                        last = min(k_hi, i + 1) if causal else k_hi     # exclusive end of the visible keys
+                        n += max(0, last - k_lo)
+            pairs[r][t] = n
+    return {"pairs": pairs,
+            "step_max": [max(pairs[r][t] for r in range(P)) for t in range(P)],
+            "rank_total": [sum(pairs[r]) for r in range(P)]}
+
+
+def balance_batches(lengths, replicas):
+    """Token-balanced short-request batches (Section 5.2 states the goal only).  Rule: take the
+    requests longest first (equal lengths in index order) and give each to the replica with the
+    fewest tokens so far (equal totals: the lowest id).  Returns (assign, tokens)."""
+    if replicas < 1 or any(x < 0 for x in lengths):
+        raise ValueError("bad arguments")
+    tokens = [0] * replicas
+    assign = [None] * len(lengths)
+    remaining = list(range(len(lengths)))
+    while remaining:
+        longest = max(lengths[i] for i in remaining)
+        i = next(i for i in remaining if lengths[i] == longest)
+        remaining.remove(i)
+        rep = tokens.index(min(tokens))
+        assign[i] = rep
+        tokens[rep] += lengths[i]
+    return assign, tokens
+
+
 def sp_volumes(s, d, n_h, n_kv, d_h, T, G):
     """Section 5.3's communication (per node) and computation (per GPU) volumes, written term by term
     with exact rational arithmetic: {(stage, strategy): (comm, comp)} for stage in ("attn", "mlp") and

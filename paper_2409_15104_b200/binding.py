@@ -13,6 +13,7 @@ PEC_OK = 0
 PEC_ERR_TIMEOUT = -6
 PEC_BF16, PEC_F32 = 1, 2
 PEC_TILE_SKIP, PEC_TILE_PARTIAL, PEC_TILE_FULL = 0, 1, 2
+PEC_LAYOUT_ZIGZAG, PEC_LAYOUT_CONTIGUOUS = 0, 1
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libpec.so")
@@ -87,7 +88,8 @@ class pec_plan(ctypes.Structure):
 
 
 EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_attn_merge_n", "pec_plan_partitions",
-           "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size", "pec_decode_attn_static", "pec_select_sp", "pec_linear")
+           "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size", "pec_decode_attn_static", "pec_select_sp", "pec_linear",
+           "pec_plan_ring", "pec_balance_batches")
 PEC_DECODE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 PEC_MERGE_MAX_PARTS = 16
 
@@ -127,6 +129,13 @@ def load():
                                ctypes.c_void_p]
     lib.pec_select_sp.restype = ctypes.c_int
     lib.pec_select_sp.argtypes = [ctypes.POINTER(pec_sp_inputs), ctypes.POINTER(pec_sp_choice)]
+    lib.pec_plan_ring.restype = ctypes.c_int
+    lib.pec_plan_ring.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                  ctypes.POINTER(ctypes.c_int64), ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
+                                  ctypes.POINTER(ctypes.c_int64), ctypes.c_int64]
+    lib.pec_balance_batches.restype = ctypes.c_int
+    lib.pec_balance_batches.argtypes = [ctypes.POINTER(ctypes.c_int32), ctypes.c_int32, ctypes.c_int32,
+                                        ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)]
     lib.pec_last_error.restype = ctypes.c_char_p
     lib.pec_last_error.argtypes = []
     _lib = lib
@@ -374,3 +383,28 @@ def pec_plan_partitions(seq_len, num_parts, chunk_len=0, align=128, block_m=128,
         "chunks": [(int(cs[c]), int(cl[c])) for c in range(nch)],
         "nq_tiles": int(plan.nq_tiles), "nk_tiles": int(plan.nk_tiles), "tile_class": tc,
     }
+
+
+def pec_plan_ring(seq_len, num_parts, align=128, layout=PEC_LAYOUT_ZIGZAG, causal=True):
+    """Ring-attention work plan (see include/pec.h): pairs[r][t], step_max[t], rank_total[r] as Python ints."""
+    lib = load()
+    P = num_parts
+    pairs = (ctypes.c_int64 * max(P * P, 1))()
+    step_max = (ctypes.c_int64 * max(P, 1))()
+    rank_total = (ctypes.c_int64 * max(P, 1))()
+    _check(lib.pec_plan_ring(seq_len, num_parts, align, layout, 1 if causal else 0, pairs, max(P * P, 1),
+                             step_max, rank_total, max(P, 1)))
+    return {"pairs": [[int(pairs[r * P + t]) for t in range(P)] for r in range(P)],
+            "step_max": [int(step_max[t]) for t in range(P)],
+            "rank_total": [int(rank_total[r]) for r in range(P)]}
+
+
+def pec_balance_batches(lengths, replicas):
+    """Token-balanced assignment of short requests to replicas (see include/pec.h): (assign, tokens)."""
+    lib = load()
+    n = len(lengths)
+    arr = (ctypes.c_int32 * max(n, 1))(*lengths)
+    assign = (ctypes.c_int32 * max(n, 1))()
+    tokens = (ctypes.c_int64 * max(replicas, 1))()
+    _check(lib.pec_balance_batches(arr, n, replicas, assign, tokens))
+    return [int(assign[i]) for i in range(n)], [int(tokens[r]) for r in range(replicas)]

@@ -2,6 +2,8 @@
 // Integer arithmetic only; the rule is stated in pec.h.  The paper asks for segments handled
 // by different replicas (Section 2.2) and for prefills that pause between kernels
 // (Section 5.1); pairing block p with block 2P-1-p equalises the causal work per partition.
+#include <algorithm>
+#include <vector>
 #include "pec_internal.h"
 
 namespace pec {
@@ -103,6 +105,95 @@ extern "C" int pec_plan_partitions(int64_t seq_len, int32_t num_parts, int64_t c
             }
         }
     }
+    return PEC_OK;
+}
+
+// Visible (query, key) pairs between query rows [a, b) and keys [c, d): a key j counts for row i
+// when j <= i (causal) or always.  Rows below the first key see nothing, rows i in [c, d-1) see
+// i + 1 - c keys (an arithmetic series), rows from d - 1 on see all d - c.
+static __int128 interval_pairs(int64_t a, int64_t b, int64_t c, int64_t d, bool causal)
+{
+    if (b <= a || d <= c) return 0;
+    const __int128 n = d - c;
+    if (!causal) return (__int128)(b - a) * n;
+    __int128 total = 0;
+    const int64_t lo1 = a > c ? a : c, hi1 = b < d - 1 ? b : d - 1;
+    if (hi1 > lo1) {
+        const __int128 m = hi1 - lo1;
+        total += m * (lo1 + 1 - c) + m * (m - 1) / 2;
+    }
+    const int64_t lo2 = a > d - 1 ? a : d - 1;
+    if (b > lo2) total += (__int128)(b - lo2) * n;
+    return total;
+}
+
+// The (up to two) row intervals of ring rank r under a layout.
+static int rank_intervals(int64_t seq_len, int32_t num_parts, int32_t r, int32_t align, int32_t layout,
+                          int64_t lo[2], int64_t hi[2])
+{
+    if (layout == PEC_LAYOUT_ZIGZAG) { zigzag_intervals(seq_len, num_parts, r, align, lo, hi); return 2; }
+    const int64_t units = ceil_div(seq_len, align);
+    lo[0] = bound_at(r, units, num_parts, align, seq_len);
+    hi[0] = bound_at((int64_t)r + 1, units, num_parts, align, seq_len);
+    lo[1] = hi[1] = 0;
+    return 1;
+}
+
+extern "C" int pec_plan_ring(int64_t seq_len, int32_t num_parts, int32_t align, int32_t layout, int32_t causal,
+                             int64_t *pairs, int64_t pairs_cap, int64_t *step_max, int64_t *rank_total, int64_t vec_cap)
+{
+    if (seq_len < 0 || num_parts < 1 || align < 1 || (layout != PEC_LAYOUT_ZIGZAG && layout != PEC_LAYOUT_CONTIGUOUS)) {
+        set_error("pec_plan_ring: need seq_len >= 0, num_parts >= 1, align >= 1 and a known layout");
+        return PEC_ERR_INVALID_ARG;
+    }
+    const int64_t P = num_parts;
+    if ((pairs && pairs_cap < P * P) || ((step_max || rank_total) && vec_cap < P)) {
+        set_error("pec_plan_ring: a caller array is smaller than the count it must hold");
+        return PEC_ERR_CAPACITY;
+    }
+    for (int64_t t = 0; t < P; ++t) {
+        if (step_max) step_max[t] = 0;
+        if (rank_total) rank_total[t] = 0;
+    }
+    for (int32_t r = 0; r < num_parts; ++r) {
+        int64_t qlo[2], qhi[2];
+        const int nq = rank_intervals(seq_len, num_parts, r, align, layout, qlo, qhi);
+        for (int32_t t = 0; t < num_parts; ++t) {
+            const int32_t src = (int32_t)(((int64_t)r - t + P) % P);
+            int64_t klo[2], khi[2];
+            const int nk = rank_intervals(seq_len, num_parts, src, align, layout, klo, khi);
+            __int128 total = 0;
+            for (int a = 0; a < nq; ++a)
+                for (int b = 0; b < nk; ++b) total += interval_pairs(qlo[a], qhi[a], klo[b], khi[b], causal != 0);
+            const int64_t v = (int64_t)total;
+            if (pairs) pairs[(int64_t)r * P + t] = v;
+            if (step_max && v > step_max[t]) step_max[t] = v;
+            if (rank_total) rank_total[r] += v;
+        }
+    }
+    return PEC_OK;
+}
+
+extern "C" int pec_balance_batches(const int32_t *lengths, int32_t n, int32_t replicas, int32_t *assign, int64_t *tokens)
+{
+    if (n < 0 || replicas < 1 || (n > 0 && (!lengths || !assign))) {
+        set_error("pec_balance_batches: need n >= 0, replicas >= 1 and non-NULL lengths/assign");
+        return PEC_ERR_INVALID_ARG;
+    }
+    for (int32_t i = 0; i < n; ++i)
+        if (lengths[i] < 0) { set_error("pec_balance_batches: request %d has a negative length", (int)i); return PEC_ERR_INVALID_ARG; }
+    std::vector<int32_t> order((size_t)n);
+    for (int32_t i = 0; i < n; ++i) order[(size_t)i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return lengths[x] > lengths[y]; });
+    std::vector<int64_t> load((size_t)replicas, 0);
+    for (int32_t i : order) {
+        int32_t best = 0;
+        for (int32_t rep = 1; rep < replicas; ++rep)
+            if (load[(size_t)rep] < load[(size_t)best]) best = rep;
+        assign[i] = best;
+        load[(size_t)best] += lengths[i];
+    }
+    if (tokens) for (int32_t rep = 0; rep < replicas; ++rep) tokens[rep] = load[(size_t)rep];
     return PEC_OK;
 }
 

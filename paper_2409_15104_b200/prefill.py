@@ -7,6 +7,8 @@ Orchestration only (which call, which buffer): all arithmetic happens inside lib
 * chunked_prefill     - a long prefill cut into preemptible chunks, each resumed from the
   stored K/V prefix (the pause points fall between kernel launches).
 * varlen_prefill      - a packed batch of short requests.
+* ring_prefill        - ring-attention sequence parallelism with every rank emulated on one GPU:
+  rank r keeps the query rows of its own zigzag segment and meets one K/V segment per ring step.
 """
 import torch
 
@@ -124,3 +126,44 @@ def chunked_prefill(q, k, v, chunk_len, o, lse, stream=None, between_chunks=None
 def varlen_prefill(q, k, v, cu_seqlens, o=None, lse=None, stream=None):
     """Packed batch of short causal prefills (cu_seqlens: int32 CUDA tensor [B+1])."""
     return binding.pec_prefill_attn(q, k, v, cu_seqlens=cu_seqlens, causal=True, o=o, lse=lse, stream=stream)
+
+
+def ring_prefill(q, k, v, num_parts, part_align=128, stream=None):
+    """The P x P (rank, ring step) launches of ring-attention SP (Section 2.2) on one GPU, no rank
+    waiting for another: rank r owns the query rows of zigzag partition r and at step t attends to
+    the keys of partition (r - t) mod P; each rank merges its P partials through their LSE.
+    Returns (o [S,Hq,128] in the input dtype, lse [S,Hq] fp32, launches)."""
+    S, Hq = q.shape[0], q.shape[1]
+    P = num_parts
+    plan = binding.pec_plan_partitions(S, P, 0, part_align, 128, 128, True, tiles=False)
+    f32 = torch.float32
+    out_o = torch.empty((S, Hq, 128), dtype=q.dtype, device=q.device)
+    out_l = torch.empty((S, Hq), dtype=f32, device=q.device)
+    longest = max((hi - lo for ivs in plan["parts"] for lo, hi in ivs), default=0)
+    run_o = torch.empty((max(longest, 1), Hq, 128), dtype=f32, device=q.device)
+    run_l = torch.empty((max(longest, 1), Hq), dtype=f32, device=q.device)
+    tmp_o, tmp_l = torch.empty_like(run_o), torch.empty_like(run_l)
+    launches = 0
+    for r in range(P):
+        for lo, hi in plan["parts"][r]:
+            n = hi - lo
+            if n <= 0:
+                continue
+            for t in range(P):
+                first, last = t == 0, t == P - 1
+                direct = first and last                       # one rank: the partial is the result
+                o = out_o[lo:hi] if direct else (run_o[:n] if first else tmp_o[:n])
+                l = out_l[lo:hi] if direct else (run_l[:n] if first else tmp_l[:n])
+                binding.pec_prefill_attn(q, k, v, seq_len=S, chunk_start=lo, chunk_len=n, kv_len=S,
+                                         part_id=(r - t) % P, num_parts=P, part_align=part_align, causal=True,
+                                         o=o, lse=l, stream=stream)
+                launches += 1
+                if first:
+                    continue
+                if last:
+                    binding.pec_attn_merge(run_o[:n], run_l[:n], tmp_o[:n], tmp_l[:n], o_out=out_o[lo:hi],
+                                           lse_out=out_l[lo:hi], stream=stream)
+                else:
+                    binding.pec_attn_merge(run_o[:n], run_l[:n], tmp_o[:n], tmp_l[:n], inplace=True, stream=stream)
+                launches += 1
+    return out_o, out_l, launches

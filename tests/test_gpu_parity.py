@@ -339,3 +339,19 @@ def test_attention_layer_steps_chain_through_strides(pec):
     want = oracle.prefill_attn(q.cpu(), k.cpu(), v.cpu(), seq_len=T)
     compare(o, lse, *want, 2e-2, 1e-3, "attention on projected q, k, v")
     assert np.abs(out.float().cpu().double().numpy() - oracle.linear(o.view(T, hq * 128).cpu(), w_l)).max() <= 2e-2
+
+
+# ------------------------------------------------------------------ ring-attention step form
+@pytest.mark.parametrize("S,P,hq,hkv", [(2048, 4, 4, 2), (1500, 3, 2, 1), (700, 1, 2, 2), (300, 8, 2, 1)])
+def test_ring_prefill_every_rank_and_step_equals_monolithic(pec, S, P, hq, hkv):
+    from paper_2409_15104_b200 import prefill
+    q, k, v = _qkv(workloads.BASE_SEED + 70 + P, S, hq, hkv, torch.bfloat16)
+    o, lse, launches = prefill.ring_prefill(*_gpu(q, k, v), num_parts=P, part_align=64)
+    pec.check_status()
+    want_o, want_l = oracle.prefill_attn(q, k, v, seq_len=S)
+    compare(o, lse, want_o, want_l, *TOL[torch.bfloat16], f"ring S={S} P={P}")
+    # one attention launch per (rank interval, step) and one merge per step after the first
+    ivs = sum(1 for part in pec.pec_plan_partitions(S, P, 0, 64, 128, 128, True, tiles=False)["parts"] for lo, hi in part if hi > lo)
+    assert launches == ivs * (2 * P - 1)
+    # the plan's per-step work adds up to the causal total the launches computed
+    assert sum(pec.pec_plan_ring(S, P, 64)["rank_total"]) == S * (S + 1) // 2

@@ -15,6 +15,7 @@ import oracle.reference as ref
 import test_oracle_pins as pins
 import test_oracle_planner as plan_pins
 import test_sp_cost_model as sp_pins
+import test_ring_and_batches as ring_pins
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ORACLE_DIR = os.path.join(os.path.dirname(HERE), "oracle")
@@ -60,7 +61,8 @@ def _some_pin_fails(calls):
 def _all_oracle_pins():
     # of the cost-model tests only the two that pin the oracle itself (the others compare the library with it)
     return (_pin_calls(pins) + _pin_calls(plan_pins) +
-            [sp_pins.test_oracle_volumes_match_the_hand_worked_example, sp_pins.test_oracle_limiting_cases])
+            [sp_pins.test_oracle_volumes_match_the_hand_worked_example, sp_pins.test_oracle_limiting_cases] +
+            _pin_calls(ring_pins))
 
 
 def test_the_unmutated_oracle_passes_every_pin():
@@ -116,6 +118,11 @@ PY_MUTATIONS = {
     "Megatron attention term not divided by T": ("qkv / T + 4 * (s * T) ** 2 * d / T + out_proj", "qkv / T + 4 * (s * T) ** 2 * d + out_proj"),
     "Ulysses all-to-all counts G not G-1": ("a2a = 2 * s * (n_h + n_kv) * d_h * (G - 1)", "a2a = 2 * s * (n_h + n_kv) * d_h * G"),
     "linear without the transpose of w": ('@ _as_f32(w).astype(np.float64).T', '@ _as_f32(w).astype(np.float64)[:, ::-1].T'),
+    "ring sends the keys the other way round": ("keys = seg[(r - t) % P]", "keys = seg[(r + t) % P]"),
+    "ring step forgets the diagonal key": ("last = min(k_hi, i + 1) if causal else k_hi", "last = min(k_hi, i) if causal else k_hi"),
+    "contiguous segments cut like zigzag blocks": ("b = [min(S, align * ((k * U) // P)) for k in range(P + 1)]", "b = [min(S, align * ((k * U) // (2 * P))) for k in range(P + 1)]"),
+    "batches built shortest first": ("longest = max(lengths[i] for i in remaining)", "longest = min(lengths[i] for i in remaining)"),
+    "batch goes to the fullest replica": ("rep = tokens.index(min(tokens))", "rep = tokens.index(max(tokens))"),
     "MLP parameter volume 4 d^2": ("(8 * d * d * (T - 1) * G / T, 16 * s * d * d)", "(4 * d * d * (T - 1) * G / T, 16 * s * d * d)"),
 }
 
@@ -130,6 +137,15 @@ def test_a_mistake_in_the_python_oracle_is_caught(name, monkeypatch):
     mod.__file__ = ref.__file__
     exec(compile(src.replace(old, new), "reference_mutant.py", "exec"), mod.__dict__)
     for attr in ("attn_rows", "prefill_attn", "varlen_attn", "merge", "merge_n", "plan_partitions",
-                 "partition_intervals", "sp_volumes", "select_sp", "linear"):
+                 "partition_intervals", "sp_volumes", "select_sp", "linear", "plan_ring", "ring_segments",
+                 "balance_batches"):
         monkeypatch.setattr(oracle, attr, getattr(mod, attr))
+    # The ring/batch pin file also compares the library with the oracle; here the library is replaced by an
+    # echo of the mutant, so that only the pins proper (enumeration, hand-worked values, bounds) can object.
+    names = {v: k for k, v in ring_pins.LAYOUTS.items()}
+    echo = types.SimpleNamespace(
+        pec_plan_ring=lambda S, P, align=128, layout=0, causal=True: mod.plan_ring(S, P, align, names[layout], causal),
+        pec_balance_batches=lambda lengths, replicas: mod.balance_batches(lengths, replicas),
+        PecError=ValueError, PEC_LAYOUT_ZIGZAG=0, PEC_LAYOUT_CONTIGUOUS=1)
+    monkeypatch.setattr(ring_pins, "binding", echo)
     assert _some_pin_fails(_all_oracle_pins()), f"no pin noticed: {name}"
