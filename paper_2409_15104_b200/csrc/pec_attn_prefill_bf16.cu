@@ -65,7 +65,7 @@ struct Geom {
 };
 
 struct Shared {
-    uint64_t bar_q;
+    uint64_t bar_q[2];                       // one per stage's Q tile
     uint64_t kv_full[kStages], kv_empty[kStages];
     uint64_t s_full[2], s_taken[2], p_ready[2];   // [stage], one phase per key tile
     uint64_t pv_done[2];                     // one phase per PV product of the stage
@@ -105,12 +105,15 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.y, kvh = h / p.group;
 
-    // Thread 0 works out the CTA's geometry: heaviest (latest) causal tiles first; per stage the
-    // rows, positions and number of key tiles it takes part in.  Key tiles are walked interval 0
+    // The loader thread works out the CTA's geometry: heaviest (latest) causal tiles first; per stage
+    // the rows, positions and number of key tiles it takes part in.  Key tiles are walked interval 0
     // first, then interval 1, in ascending position, so each stage's tiles are a prefix of the walk.
-    // The set-up runs in parallel: warp 1 initialises the barriers and prefetches the tensor maps,
-    // warp 2 allocates tensor memory, thread 0 works out the geometry.
-    if (tid == 0) {
+    // It then initialises the barriers its loads complete on and starts the first loads (Q of stage 0,
+    // K(0), Q of stage 1, V(0)) before the CTA-wide sync: their latency is the longest part of a CTA's
+    // start-up.  Meanwhile warp 1 initialises the other barriers and warp 2 allocates tensor memory.
+    // (Loops over the two intervals and stages are unrolled with constant indices, so the geometry
+    // stays in registers.)
+    if (tid == kLoadWarp * 32) {
         Geom g = {};
         TileJob job;
         g.found = locate_tile(p, (int64_t)gridDim.x - 1 - blockIdx.x, kBlockM, job) ? 1 : 0;
@@ -118,7 +121,13 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         if (g.found) {
             g.q_row0 = (int32_t)job.q_row0; g.out_row0 = (int32_t)job.out_row0; g.kv_row0 = (int32_t)job.kv_row0;
             g.cnt[0] = g.cnt[1] = 0;
-            for (int t = 0; t < 2; ++t) { g.lo[t] = (int32_t)job.iv_lo[t]; g.hi[t] = (int32_t)job.iv_hi[t]; }
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const bool used = t < job.n_iv;
+                g.lo[t] = used ? (int32_t)job.iv_lo[t] : 0;
+                g.hi[t] = used ? (int32_t)job.iv_hi[t] : 0;
+            }
+#pragma unroll
             for (int st = 0; st < 2; ++st) {
                 int32_t rows = job.n_rows - st * kTile;
                 rows = rows < 0 ? 0 : (rows > kTile ? kTile : rows);
@@ -127,7 +136,8 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 g.n[st] = 0;
                 if (rows > 0) {
                     const int32_t last = g.pos0[st] + rows - 1;
-                    for (int t = 0; t < job.n_iv; ++t) {
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
                         int32_t end = g.hi[t];
                         if (p.causal && end > last + 1) end = last + 1;
                         const int32_t c = end > g.lo[t] ? (end - g.lo[t] + kTile - 1) / kTile : 0;
@@ -139,10 +149,29 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             g.n_max = g.cnt[0] + g.cnt[1];
         }
         sh->g = g;                                            // a CTA past the last tile has no rows and no keys
+        mbar_init(smem_u32(&sh->bar_q[0]), 1);
+        mbar_init(smem_u32(&sh->bar_q[1]), 1);
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->kv_full[s]), 1); mbar_init(smem_u32(&sh->kv_empty[s]), 2); }
+        mbar_init_fence();
+        if (g.n_max > 0) {
+            const int krow = g.kv_row0 + (g.cnt[0] > 0 ? g.lo[0] : g.lo[1]);
+#pragma unroll
+            for (int st = 0; st < 2; ++st) {
+                const uint32_t bar_q = smem_u32(&sh->bar_q[st]);
+                mbar_arrive_expect_tx(bar_q, kTileBytes);
+                tma_load_3d(sQ + st * kTileBytes, &tm_q, bar_q, 0, h, g.q_row0 + st * kTile);
+                tma_load_3d(sQ + st * kTileBytes + kHalfTileBytes, &tm_q, bar_q, 64, h, g.q_row0 + st * kTile);
+                // ring items 0 and 1: K(0) and V(0)
+                const void *map = st ? (const void *)&tm_v : (const void *)&tm_k;
+                const uint32_t dst = sRing + st * kTileBytes, bar = smem_u32(&sh->kv_full[st]);
+                mbar_arrive_expect_tx(bar, kTileBytes);
+                tma_load_3d(dst, map, bar, 0, kvh, krow);
+                tma_load_3d(dst + kHalfTileBytes, map, bar, 64, kvh, krow);
+            }
+        }
     } else if (tid == 32) {
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
-        mbar_init(smem_u32(&sh->bar_q), 1);
-        for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&sh->kv_full[s]), 1); mbar_init(smem_u32(&sh->kv_empty[s]), 2); }
         for (int st = 0; st < 2; ++st) {
             mbar_init(smem_u32(&sh->s_full[st]), 1);
             mbar_init(smem_u32(&sh->s_taken[st]), 4);         // one arrival per softmax warp
@@ -166,15 +195,7 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         // ------------------------------------------------------------------ TMA loader
         reg_dealloc<kLightRegs>();
         if (lane == 0 && n_max > 0) {
-            const uint32_t bar_q = smem_u32(&sh->bar_q);
-            mbar_arrive_expect_tx(bar_q, 2 * kTileBytes);
-#pragma unroll
-            for (int st = 0; st < 2; ++st) {
-                const int row = sh->g.q_row0 + st * kTile;
-                tma_load_3d(sQ + st * kTileBytes, &tm_q, bar_q, 0, h, row);
-                tma_load_3d(sQ + st * kTileBytes + kHalfTileBytes, &tm_q, bar_q, 64, h, row);
-            }
-            for (int i = 0; i < 2 * n_max; ++i) {              // items: K(0), V(0), K(1), V(1), ...
+            for (int i = 2; i < 2 * n_max; ++i) {              // items: K(0), V(0) (loaded above), K(1), V(1), ...
                 const int slot = i % kStages, fill = i / kStages;
                 if (sh->abort_flag) break;
                 if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p.status)) break;
@@ -251,7 +272,7 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 return got;
             };
 
-            bool ok = wait_u(&sh->bar_q, 0) && kv_wait(0);
+            bool ok = wait_u(&sh->bar_q[st], 0) && kv_wait(0);
             if (ok) {
                 if (n_st > 0) { ok = wait_buffer(0); if (ok) issue_qk(0); }
                 kv_release(0);
@@ -402,7 +423,7 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         // conflicts) and writes it out two rows per instruction, 256 contiguous bytes each.
         if (ok && n_hf > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->o_final[st]), 0, sh, p.status));
         // A stage without keys never waited for its Q tile: the load must have landed before the tile is reused.
-        if (ok && n_hf == 0 && n_max > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->bar_q), 0, sh, p.status));
+        if (ok && n_hf == 0 && n_max > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->bar_q[st]), 0, sh, p.status));
         if (ok && sh->g.rows[st] > 0) {
             tc_fence_after();
             const bool empty = (l_run == 0.f);

@@ -27,7 +27,8 @@ __device__ __forceinline__ bool locate_tile(const AttnParams &p, int64_t tile, i
         job.n_rows = (int32_t)((p.chunk_len - r0) < block_m ? (p.chunk_len - r0) : block_m);
         job.kv_row0 = 0;
         job.n_iv = p.n_iv;
-        for (int t = 0; t < 2; ++t) { job.iv_lo[t] = p.iv_lo[t]; job.iv_hi[t] = p.iv_hi[t]; }
+        job.iv_lo[0] = p.iv_lo[0]; job.iv_hi[0] = p.iv_hi[0];
+        job.iv_lo[1] = p.iv_lo[1]; job.iv_hi[1] = p.iv_hi[1];
         return true;
     }
     int64_t t = tile;
