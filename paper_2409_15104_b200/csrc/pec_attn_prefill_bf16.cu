@@ -105,7 +105,7 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.y, kvh = h / p.group;
 
-    // The loader thread works out the CTA's geometry: heaviest (latest) causal tiles first; per stage
+    // The loader warp finds the CTA's tile and its first lane works out the geometry: heaviest (latest) causal tiles first; per stage
     // the rows, positions and number of key tiles it takes part in.  Key tiles are walked interval 0
     // first, then interval 1, in ascending position, so each stage's tiles are a prefix of the walk.
     // It then initialises the barriers its loads complete on and starts the first loads (Q of stage 0,
@@ -113,10 +113,12 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     // start-up.  Meanwhile warp 1 initialises the other barriers and warp 2 allocates tensor memory.
     // (Loops over the two intervals and stages are unrolled with constant indices, so the geometry
     // stays in registers.)
+    TileJob job;
+    bool job_found = false;
+    if (warp == kLoadWarp) job_found = locate_tile_warp(p, (int64_t)gridDim.x - 1 - blockIdx.x, kBlockM, job);   // whole warp
     if (tid == kLoadWarp * 32) {
         Geom g = {};
-        TileJob job;
-        g.found = locate_tile(p, (int64_t)gridDim.x - 1 - blockIdx.x, kBlockM, job) ? 1 : 0;
+        g.found = job_found ? 1 : 0;
         sh->abort_flag = 0;
         if (g.found) {
             g.q_row0 = (int32_t)job.q_row0; g.out_row0 = (int32_t)job.out_row0; g.kv_row0 = (int32_t)job.kv_row0;

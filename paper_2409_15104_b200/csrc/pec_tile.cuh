@@ -52,4 +52,46 @@ __device__ __forceinline__ bool locate_tile(const AttnParams &p, int64_t tile, i
     return false;
 }
 
+// The same search done by a whole converged warp: for a packed batch each lane takes every 32nd
+// request (the two table reads of all requests are in flight together instead of one dependent pair
+// per request), tile counts are prefix-summed with shuffles, and the lane that owns the tile's request
+// broadcasts it.  Every lane returns the same job.
+__device__ __forceinline__ bool locate_tile_warp(const AttnParams &p, int64_t tile, int block_m, TileJob &job)
+{
+    if (p.cu_seqlens == nullptr) return locate_tile(p, tile, block_m, job);
+    const int lane = threadIdx.x & 31;
+    int64_t before = 0;                                   // tiles of the requests in earlier groups of 32
+    for (int b0 = 0; b0 < p.B; b0 += 32) {
+        const int b = b0 + lane;
+        int64_t s = 0, e = 0;
+        if (b < p.B) { s = p.cu_seqlens[b]; e = p.cu_seqlens[b + 1]; }
+        const int64_t nt = (e - s + block_m - 1) / block_m;
+        int64_t incl = nt;                                // inclusive prefix sum over the lanes
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int64_t up = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        const bool mine = b < p.B && tile >= before + incl - nt && tile < before + incl;
+        const unsigned who = __ballot_sync(0xffffffffu, mine);
+        if (who) {
+            const int src = __ffs(who) - 1;
+            const int64_t s_b = __shfl_sync(0xffffffffu, s, src), e_b = __shfl_sync(0xffffffffu, e, src);
+            const int64_t first = __shfl_sync(0xffffffffu, before + incl - nt, src);
+            const int64_t r0 = (tile - first) * block_m;
+            job.q_row0 = s_b + r0;
+            job.out_row0 = s_b + r0;
+            job.q_pos0 = r0;
+            job.n_rows = (int32_t)((e_b - s_b - r0) < block_m ? (e_b - s_b - r0) : block_m);
+            job.kv_row0 = s_b;
+            job.n_iv = 1;
+            job.iv_lo[0] = 0; job.iv_hi[0] = e_b - s_b;
+            job.iv_lo[1] = 0; job.iv_hi[1] = 0;
+            return true;
+        }
+        before += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    return false;
+}
+
 }  // namespace pec
