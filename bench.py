@@ -31,7 +31,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) of one attention launch, from the ncu capture summarised in
 # profiles/attn_prefill_bf16_kernel_c3.md (mean of its two launches).  Valid for that kernel and workload
 # only: set an entry back to None when the kernel changes.
-NCU_TRAFFIC_BYTES = {"c3": 769.0e6}
+NCU_TRAFFIC_BYTES = {"c3": 766.5e6}
 
 
 def load_peaks():
