@@ -23,7 +23,7 @@ class PartitionedPrefill:
     degenerates to the running two-way merge.
     """
 
-    def __init__(self, seq_len, hq, num_parts, dtype, device, part_align=128, partial_budget_bytes=24 << 30):
+    def __init__(self, seq_len, hq, num_parts, dtype, device, part_align=128, partial_budget_bytes=80 << 30):
         self.S, self.Hq, self.P, self.align = seq_len, hq, num_parts, part_align
         self.dtype = dtype
         f32 = torch.float32
