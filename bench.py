@@ -32,6 +32,8 @@ NOMINAL_HBM_GBS = 8000.0
 # profiles/attn_prefill_bf16_kernel_c3.md (mean of its two launches).  Valid for that kernel and workload
 # only: set an entry back to None when the kernel changes.
 NCU_TRAFFIC_BYTES = {"c3": 766.5e6}
+# Pipe activity of the same two captured launches (percent of peak sustained, elapsed): same validity rule.
+NCU_PIPES = {"c3": {"tensor_pipe_active_pct": 61.0, "xu_pipe_pct": 61.7, "ms_per_launch_under_ncu": 0.912}}
 
 
 def load_peaks():
@@ -297,6 +299,7 @@ def run_ours(args, wl):
         "roofline": {"bound": "tensor", "kernel": "attn_prefill_bf16_kernel", "achieved": attn_tflops,
                      "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": attn_tflops / peaks["bf16_sustained"],
                      "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "traffic_unit": "bytes per launch (ncu dram read + write)",
+                     "ncu": NCU_PIPES.get(wl.name),
                      "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step)",
                      "frac_of_burst": attn_tflops / peaks["bf16_burst"], "frac_of_nominal": attn_tflops / NOMINAL_BF16_TFLOPS,
                      "flops_per_launch": flops_launch, "ms_per_launch": attn_avg_ms},

@@ -185,7 +185,9 @@ def test_row_maximum_that_moves(pec, dtype, shape):
 
 # ------------------------------------------------------------------ packed batches
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
-@pytest.mark.parametrize("lens", [[5], [128, 128], [1, 300, 0, 77, 129, 64], [200, 1, 1, 511]])
+@pytest.mark.parametrize("lens", [[5], [128, 128], [1, 300, 0, 77, 129, 64], [200, 1, 1, 511],
+                                  [(i * 37) % 200 for i in range(70)]],      # more requests than one warp-wide search step
+                         ids=["one", "two_tiles", "with_empty", "ragged", "seventy"])
 def test_varlen_batch(pec, dtype, lens):
     cu = workloads.cu_seqlens(lens)
     T = cu[-1]
