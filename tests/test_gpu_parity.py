@@ -357,3 +357,35 @@ def test_ring_prefill_every_rank_and_step_equals_monolithic(pec, S, P, hq, hkv):
     assert launches == ivs * (2 * P - 1)
     # the plan's per-step work adds up to the causal total the launches computed
     assert sum(pec.pec_plan_ring(S, P, 64)["rank_total"]) == S * (S + 1) // 2
+
+
+# ------------------------------------------------------------------ seeded random call shapes
+def _random_call(seed):
+    g = np.random.Generator(np.random.Philox(key=9000 + seed))
+    S = int(g.integers(1, 1400))
+    hkv = int(g.choice([1, 2, 4]))
+    hq = hkv * int(g.choice([1, 2, 4]))
+    P = int(g.choice([1, 1, 2, 3, 4, 8]))
+    align = int(g.choice([1, 16, 64, 128]))
+    causal = bool(g.integers(0, 4) > 0)
+    c0 = int(g.integers(0, S))
+    n = int(g.integers(1, S - c0 + 1))
+    kv_len = int(g.integers(c0 + n, S + 1)) if causal else int(g.integers(1, S + 1))
+    return dict(S=S, hq=hq, hkv=hkv, P=P, part=int(g.integers(0, P)), align=align, causal=causal, c0=c0, n=n, kv_len=kv_len)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_chunk_partition_prefix_combinations(pec, seed):
+    """Chunk start/length, K/V prefix, partition, alignment, GQA ratio and mask drawn from a seed: the two
+    stages of a CTA then see different numbers of key tiles, none at all, or a single ragged one."""
+    c = _random_call(seed)
+    q, k, v = _qkv(9100 + seed, c["S"], c["hq"], c["hkv"], torch.bfloat16)
+    want = oracle.prefill_attn(q, k, v, seq_len=c["S"], chunk_start=c["c0"], chunk_len=c["n"], kv_len=c["kv_len"],
+                               part_id=c["part"], num_parts=c["P"], part_align=c["align"], causal=c["causal"])
+    dq, dk, dv = _gpu(q, k, v)
+    dk[c["kv_len"]:] = float("nan"); dv[c["kv_len"]:] = float("nan")     # nothing past the prefix may be read
+    o, lse = pec.pec_prefill_attn(dq, dk, dv, seq_len=c["S"], chunk_start=c["c0"], chunk_len=c["n"], kv_len=c["kv_len"],
+                                  part_id=c["part"], num_parts=c["P"], part_align=c["align"], causal=c["causal"],
+                                  out_dtype=torch.float32)
+    pec.check_status()
+    compare(o, lse, *want, *TOL[torch.bfloat16], f"random call {c}")
