@@ -7,6 +7,8 @@ Orchestration only (which call, which buffer): all arithmetic happens inside lib
 * chunked_prefill     - a long prefill cut into preemptible chunks, each resumed from the
   stored K/V prefix (the pause points fall between kernel launches).
 * varlen_prefill      - a packed batch of short requests.
+* StreamedPrefill     - consecutive partitioned prefills whose inputs come from and whose results go to
+  host memory: the copies of neighbouring steps overlap the compute of the current one.
 * ring_prefill        - ring-attention sequence parallelism with every rank emulated on one GPU:
   rank r keeps the query rows of its own zigzag segment and meets one K/V segment per ring step.
 """
@@ -48,14 +50,16 @@ class PartitionedPrefill:
     def launches_per_step(self):
         return self.P + self.merge_launches()
 
-    def run(self, q, k, v, stream=None, time_kernels=False):
-        """Returns (o [S,Hq,128] in the input dtype, lse [S,Hq] fp32)."""
+    def run(self, q, k, v, stream=None, time_kernels=False, out=None):
+        """Returns (o [S,Hq,128] in the input dtype, lse [S,Hq] fp32); `out` = (o, lse) buffers to write the
+        result to instead of the runner's own."""
         P = self.P
+        out_o, out_l = (self.out_o, self.out_l) if out is None else out
         self.plan = binding.pec_plan_partitions(self.S, P, 0, self.align, 128, 128, True, tiles=False)
         self.merge_parts = []
         if P == 1:
-            self._attn(q, k, v, 0, self.out_o, self.out_l, stream, time_kernels)
-            return self.out_o, self.out_l
+            self._attn(q, k, v, 0, out_o, out_l, stream, time_kernels)
+            return out_o, out_l
         p = 0
         first = True
         while p < P:
@@ -75,17 +79,17 @@ class PartitionedPrefill:
             if len(group) == 2 and not last:
                 binding.pec_attn_merge(o_parts[0], l_parts[0], o_parts[1], l_parts[1], inplace=True, stream=stream)
             elif len(group) == 2:
-                binding.pec_attn_merge(o_parts[0], l_parts[0], o_parts[1], l_parts[1], o_out=self.out_o,
-                                       lse_out=self.out_l, stream=stream)
+                binding.pec_attn_merge(o_parts[0], l_parts[0], o_parts[1], l_parts[1], o_out=out_o,
+                                       lse_out=out_l, stream=stream)
             elif last:
-                binding.pec_attn_merge_n(o_parts, l_parts, o_out=self.out_o, lse_out=self.out_l, stream=stream)
+                binding.pec_attn_merge_n(o_parts, l_parts, o_out=out_o, lse_out=out_l, stream=stream)
             else:
                 binding.pec_attn_merge_n(o_parts, l_parts, inplace=True, stream=stream)
             if ev:
                 ev[1].record(stream)
             self.merge_parts.append(len(group))
             first = False
-        return self.out_o, self.out_l
+        return out_o, out_l
 
     def _events(self, on, store, stream):
         if not on:
@@ -167,3 +171,48 @@ def ring_prefill(q, k, v, num_parts, part_align=128, stream=None):
                     binding.pec_attn_merge(run_o[:n], run_l[:n], tmp_o[:n], tmp_l[:n], inplace=True, stream=stream)
                 launches += 1
     return out_o, out_l, launches
+
+
+class StreamedPrefill:
+    """Host-to-host pipelining of consecutive prefills run by a PartitionedPrefill: while step i computes,
+    the inputs of step i+1 are copied to the device and the result of step i-1 is copied back (three
+    streams, two sets of device input and output buffers; PCIe carries both directions at once).
+    Host tensors must be pinned.  Orchestration only: every copy is a cudaMemcpyAsync issued by torch,
+    every computation a call of the library."""
+
+    def __init__(self, runner, hkv, device):
+        self.runner = runner
+        S, Hq, dt = runner.S, runner.Hq, runner.dtype
+        self.inp = [tuple(torch.empty((S, h, 128), dtype=dt, device=device) for h in (Hq, hkv, hkv)) for _ in range(2)]
+        self.out = [(torch.empty((S, Hq, 128), dtype=dt, device=device),
+                     torch.empty((S, Hq), dtype=torch.float32, device=device)) for _ in range(2)]
+        self.s_in, self.s_comp, self.s_out = (torch.cuda.Stream(device=device) for _ in range(3))
+        self.computed = [None, None]      # event: the step that last used buffer set b has finished computing
+        self.copied_out = [None, None]    # event: its result has left the device
+        self.step = 0
+
+    def submit(self, q_h, k_h, v_h, o_h, l_h):
+        """Enqueue one prefill: q_h, k_h, v_h -> device -> (o_h, l_h).  Returns at once."""
+        b = self.step & 1
+        self.step += 1
+        with torch.cuda.stream(self.s_in):
+            if self.computed[b] is not None:
+                self.s_in.wait_event(self.computed[b])           # the inputs of two steps ago are no longer read
+            for dst, src in zip(self.inp[b], (q_h, k_h, v_h)):
+                dst.copy_(src, non_blocking=True)
+            arrived = torch.cuda.Event(); arrived.record(self.s_in)
+        with torch.cuda.stream(self.s_comp):
+            self.s_comp.wait_event(arrived)
+            if self.copied_out[b] is not None:
+                self.s_comp.wait_event(self.copied_out[b])       # the result of two steps ago has been read out
+            self.runner.run(*self.inp[b], stream=self.s_comp, out=self.out[b])
+            self.computed[b] = torch.cuda.Event(); self.computed[b].record(self.s_comp)
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.computed[b])
+            o_h.copy_(self.out[b][0], non_blocking=True)
+            l_h.copy_(self.out[b][1], non_blocking=True)
+            self.copied_out[b] = torch.cuda.Event(); self.copied_out[b].record(self.s_out)
+
+    def drain(self):
+        for s in (self.s_in, self.s_comp, self.s_out):
+            s.synchronize()

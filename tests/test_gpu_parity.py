@@ -389,3 +389,28 @@ def test_random_chunk_partition_prefix_combinations(pec, seed):
                                   out_dtype=torch.float32)
     pec.check_status()
     compare(o, lse, *want, *TOL[torch.bfloat16], f"random call {c}")
+
+
+def test_streamed_prefill_matches_one_step_at_a_time(pec):
+    """Five consecutive host-to-host steps with different inputs through the three-stream pipeline: every
+    result equals (bit for bit) what the same runner gives for that input alone."""
+    from paper_2409_15104_b200.prefill import PartitionedPrefill, StreamedPrefill
+    S, hq, hkv, P = 1536, 4, 2, 4
+    runner = PartitionedPrefill(S, hq, P, torch.bfloat16, DEV)
+    pipe = StreamedPrefill(runner, hkv, DEV)
+    steps = []
+    for i in range(5):
+        q, k, v = (t.pin_memory() for t in _qkv(workloads.BASE_SEED + 300 + i, S, hq, hkv, torch.bfloat16))
+        o_h = torch.empty((S, hq, 128), dtype=torch.bfloat16).pin_memory()
+        l_h = torch.empty((S, hq), dtype=torch.float32).pin_memory()
+        steps.append((q, k, v, o_h, l_h))
+    for st in steps:
+        pipe.submit(*st)
+    pipe.drain()
+    pec.check_status()
+    for i, (q, k, v, o_h, l_h) in enumerate(steps):
+        o, l = runner.run(*_gpu(q, k, v))
+        torch.cuda.synchronize()
+        assert torch.equal(o.cpu(), o_h) and torch.equal(l.cpu(), l_h), f"step {i}"
+    want_o, want_l = oracle.prefill_attn(steps[-1][0], steps[-1][1], steps[-1][2], seq_len=S)
+    compare(steps[-1][3], steps[-1][4], want_o, want_l, *TOL[torch.bfloat16], "streamed, last step")
