@@ -428,6 +428,41 @@ def _short_batch(wl, dev, seed_offset=0):
     return (q.to(dev), k.to(dev), v.to(dev), torch.tensor(cu, dtype=torch.int32, device=dev), cu[-1], pairs)
 
 
+def run_ring(args):
+    """Extra line: the P x P (rank, ring step) launches of ring-attention SP over c3's request, every rank
+    emulated on this GPU one after the other, beside the planner's per-step work for zigzag and contiguous
+    segments (what a real ring's step times would follow)."""
+    from paper_2409_15104_b200 import binding
+    from paper_2409_15104_b200.prefill import ring_prefill
+    wl = workloads.WORKLOADS["c3"]
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    q, k, v = (t.to(dev) for t in workloads.qkv(wl.seed, wl.seq_len, wl.hq, wl.hkv, 128, wl.dtype))
+    P = wl.num_parts
+    for _ in range(max(args.warmup, 3)):
+        _, _, launches = ring_prefill(q, k, v, P, wl.part_align)
+    torch.cuda.synchronize()
+    evs = []
+    for _ in range(min(args.steps, 20)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); ring_prefill(q, k, v, P, wl.part_align); e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    binding.check_status()
+    ms = statistics.median(a.elapsed_time(b) for a, b in evs)
+    fl = workloads.attention_flops(workloads.causal_pairs(wl.seq_len), wl.hq)
+    plans = {name: binding.pec_plan_ring(wl.seq_len, P, wl.part_align, code, True)
+             for name, code in (("zigzag", binding.PEC_LAYOUT_ZIGZAG), ("contiguous", binding.PEC_LAYOUT_CONTIGUOUS))}
+    total = workloads.causal_pairs(wl.seq_len)
+    print(json.dumps({"metric": "ring-attention SP steps of all ranks on one GPU, attention TFLOP/s (extra line, not the headline)",
+                      "value": fl / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms, "n_gpus": 1, "dtype": "bf16",
+                      "data": "synthetic", "gpu_launches_per_step": launches,
+                      "planned_ring_time_in_pairs": {name: sum(pl["step_max"]) for name, pl in plans.items()},
+                      "planned_ring_efficiency": {name: total / (P * sum(pl["step_max"])) for name, pl in plans.items()},
+                      "config": {"workload": f"ring: {wl.note}; rank r's query blocks against the keys of rank (r-t) mod P",
+                                 "ranks": P, "l2": "inputs and partials exceed the 126 MB L2"}}), flush=True)
+
+
 def run_short_batch(args, wl):
     """Extra line: the packed short-request batch (c2) alone."""
     from paper_2409_15104_b200 import binding
@@ -525,7 +560,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode", "linear"], default="c3")
+    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode", "linear", "ring"], default="c3")
     ap.add_argument("--reference-seconds", type=float, default=0.0,
                     help="--impl reference: CPU seconds per step (default: 90 s spread over the steps, 0.15-20 s each)")
     ap.add_argument("--profile", action="store_true",
@@ -537,6 +572,9 @@ def main():
         return
     if args.workload == "linear":
         run_linear(args)
+        return
+    if args.workload == "ring":
+        run_ring(args)
         return
     wl = workloads.WORKLOADS[args.workload]
     if args.workload == "c2":
