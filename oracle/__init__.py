@@ -13,6 +13,8 @@ from .reference import (  # noqa: F401
     select_sp,
     linear,
     plan_partitions,
+    plan_worklist,
+    partition_rows,
     plan_ring,
     ring_segments,
     balance_batches,

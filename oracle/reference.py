@@ -111,6 +111,37 @@ def plan_partitions(seq_len, num_parts, chunk_len, align, block_m, block_n, caus
     }
 
 
+def plan_worklist(cu_seqlens, block_m, block_n, causal):
+    """Tile list of a packed batch of short requests (Section 5.2), heaviest first.
+
+    Every request is cut into tiles of block_m query rows from its own first row.  A tile's weight is
+    the number of block_n-key tiles of its request that hold at least one key some row of the tile can
+    see: with the causal mask the tile's last row, at position e - 1, sees keys [0, e), so
+    ceil(e / block_n); without it every row sees all L keys.  Entries (first row of the request, position
+    of the tile's first row, rows, request length) are ordered by weight descending, then request index,
+    then position."""
+    cu = [int(x) for x in cu_seqlens]
+    entries = []
+    for b in range(len(cu) - 1):
+        L = cu[b + 1] - cu[b]
+        if L < 0:
+            raise ValueError("cu_seqlens decreases")
+        for pos0 in range(0, L, block_m):
+            n = min(block_m, L - pos0)
+            weight = _ceil_div(pos0 + n if causal else L, block_n)
+            entries.append((-weight, b, pos0, (cu[b], pos0, n, L)))
+    entries.sort(key=lambda e: e[:3])
+    return [e[3] for e in entries]
+
+
+def partition_rows(seq_len, num_parts, part_id, align, chunk_start=0, chunk_len=None):
+    """Positions of the chunk's rows that lie in zigzag partition part_id (ascending)."""
+    S = int(seq_len)
+    chunk_len = S - chunk_start if chunk_len is None else int(chunk_len)
+    ivs = plan_partitions(S, num_parts, 0, align, 1, 1, True, tiles=False)["parts"][part_id]
+    return [i for lo, hi in ivs for i in range(max(lo, chunk_start), min(hi, chunk_start + chunk_len))]
+
+
 def partition_intervals(seq_len, num_parts, part_id, align, kv_len=None):
     """Key intervals of one partition, cut to the available K/V prefix [0, kv_len)."""
     S, P, p = int(seq_len), int(num_parts), int(part_id)

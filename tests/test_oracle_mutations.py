@@ -16,6 +16,7 @@ import test_oracle_pins as pins
 import test_oracle_planner as plan_pins
 import test_sp_cost_model as sp_pins
 import test_ring_and_batches as ring_pins
+import test_worklist_planner as wl_pins
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ORACLE_DIR = os.path.join(os.path.dirname(HERE), "oracle")
@@ -62,7 +63,9 @@ def _all_oracle_pins():
     # of the cost-model tests only the two that pin the oracle itself (the others compare the library with it)
     return (_pin_calls(pins) + _pin_calls(plan_pins) +
             [sp_pins.test_oracle_volumes_match_the_hand_worked_example, sp_pins.test_oracle_limiting_cases] +
-            _pin_calls(ring_pins))
+            _pin_calls(ring_pins) +
+            _expand(wl_pins.test_worklist_covers_every_row_once_heaviest_first) + _expand(wl_pins.test_partition_rows_split_the_chunk) +
+            [wl_pins.test_worklist_hand_worked_example, wl_pins.test_worklist_ties_keep_request_then_position_order])
 
 
 def test_the_unmutated_oracle_passes_every_pin():
@@ -123,6 +126,11 @@ PY_MUTATIONS = {
     "contiguous segments cut like zigzag blocks": ("b = [min(S, align * ((k * U) // P)) for k in range(P + 1)]", "b = [min(S, align * ((k * U) // (2 * P))) for k in range(P + 1)]"),
     "batches built shortest first": ("longest = max(lengths[i] for i in remaining)", "longest = min(lengths[i] for i in remaining)"),
     "batch goes to the fullest replica": ("rep = tokens.index(min(tokens))", "rep = tokens.index(max(tokens))"),
+    "work-list weight from the tile's first row": ("weight = _ceil_div(pos0 + n if causal else L, block_n)", "weight = _ceil_div(pos0 + 1 if causal else L, block_n)"),
+    "work-list lightest first": ("entries.append((-weight, b, pos0, (cu[b], pos0, n, L)))", "entries.append((weight, b, pos0, (cu[b], pos0, n, L)))"),
+    "work-list ties by position before request": ("entries.sort(key=lambda e: e[:3])", "entries.sort(key=lambda e: (e[0], e[2], e[1]))"),
+    "work-list last tile not cut": ("n = min(block_m, L - pos0)", "n = block_m"),
+    "partition rows ignore the chunk start": ("range(max(lo, chunk_start), min(hi, chunk_start + chunk_len))", "range(lo, min(hi, chunk_start + chunk_len))"),
     "MLP parameter volume 4 d^2": ("(8 * d * d * (T - 1) * G / T, 16 * s * d * d)", "(4 * d * d * (T - 1) * G / T, 16 * s * d * d)"),
 }
 
@@ -138,7 +146,7 @@ def test_a_mistake_in_the_python_oracle_is_caught(name, monkeypatch):
     exec(compile(src.replace(old, new), "reference_mutant.py", "exec"), mod.__dict__)
     for attr in ("attn_rows", "prefill_attn", "varlen_attn", "merge", "merge_n", "plan_partitions",
                  "partition_intervals", "sp_volumes", "select_sp", "linear", "plan_ring", "ring_segments",
-                 "balance_batches"):
+                 "balance_batches", "plan_worklist", "partition_rows"):
         monkeypatch.setattr(oracle, attr, getattr(mod, attr))
     # The ring/batch pin file also compares the library with the oracle; here the library is replaced by an
     # echo of the mutant, so that only the pins proper (enumeration, hand-worked values, bounds) can object.
