@@ -28,12 +28,35 @@ from paper_2409_15104_b200 import workloads
 METRIC = "causal prefill attention TFLOP/s (tokens/s and % of dense BF16 peak alongside), 1 B200"
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (read + write) of one attention launch, from the ncu capture summarised in
-# profiles/attn_prefill_bf16_kernel_c3.md (mean of its two launches).  Valid for that kernel and workload
-# only: set an entry back to None when the kernel changes.
-NCU_TRAFFIC_BYTES = {"c3": 766.5e6}
-# Pipe activity of the same two captured launches (percent of peak sustained, elapsed): same validity rule.
-NCU_PIPES = {"c3": {"tensor_pipe_active_pct": 61.0, "xu_pipe_pct": 61.7, "ms_per_launch_under_ncu": 0.912}}
+KERNEL_SOURCES = ("pec_attn_prefill_bf16.cu", "pec_sm100.cuh", "pec_tile.cuh")
+
+
+def kernel_source_hash():
+    """First 16 hex digits of the SHA-256 over the attention kernel's sources: ties a stored profiler
+    counter to the kernel revision it was taken on."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        h.update(open(os.path.join(ROOT, "paper_2409_15104_b200", "csrc", name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def stored_counters(workload):
+    """Profiler counters of one attention launch of `workload`, read from profiles/attn_counters.txt (taken
+    offline with ncu, never in this run).  Returns None when there is no line for the workload, and marks the
+    record stale - traffic null - when the kernel sources have changed since the capture."""
+    path = os.path.join(ROOT, "profiles", "attn_counters.txt")
+    if not os.path.exists(path):
+        return None
+    for ln in open(path):
+        f = ln.split()
+        if len(f) >= 6 and not ln.startswith("#") and f[0] == workload:
+            rec = {"captured_offline": True, "kernel_source_hash_at_capture": f[1], "dram_bytes_per_launch": float(f[2]),
+                   "tensor_pipe_active_pct": float(f[3]), "xu_pipe_pct": float(f[4]), "ms_per_launch_under_ncu": float(f[5]),
+                   "note": " ".join(f[6:])}
+            rec["stale"] = rec["kernel_source_hash_at_capture"] != kernel_source_hash()
+            return rec
+    return None
 
 
 def load_peaks():
@@ -217,7 +240,7 @@ def run_ours(args, wl):
     clocks = sampler.stop() if rank == 0 else None
     binding.check_status()
     attn_ms = [a.elapsed_time(b) for a, b in runner.attn_events]
-    merge_ms = [a.elapsed_time(b) for a, b in runner.merge_events]
+    launches_per_step = runner.launches_per_step()
 
     if args.profile:
         if rank == 0:
@@ -225,7 +248,6 @@ def run_ours(args, wl):
             print(json.dumps({"profile_run": True, "ms_per_step": total_ms / args.steps,
                               "attn_ms_per_launch": sum(attn_ms) / len(attn_ms),
                               "attn_tflops": fl / wl.num_parts / (sum(attn_ms) / len(attn_ms)) / 1e9,
-                              "merge_ms_per_launch": (sum(merge_ms) / len(merge_ms)) if merge_ms else None,
                               "clocks": clocks}), flush=True)
         if dist is not None:
             dist.destroy_process_group()
@@ -248,7 +270,7 @@ def run_ours(args, wl):
     serial_step()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    serial_steps = max(1, min(args.steps, 3))
+    serial_steps = max(1, min(args.steps, 3 if wl.seq_len <= 65536 else 1))
     e0.record(stream)
     for _ in range(serial_steps):
         serial_step()
@@ -261,7 +283,7 @@ def run_ours(args, wl):
     pipe.submit(q_h, k_h, v_h, o_h, l_h)
     pipe.drain()
     barrier()
-    e2e_steps = max(1, min(args.steps, 20))
+    e2e_steps = max(1, min(args.steps, 20 if wl.seq_len <= 65536 else 4))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(pipe.s_in)                                       # nothing is in flight: first operation of the region
     for _ in range(e2e_steps):
@@ -286,23 +308,39 @@ def run_ours(args, wl):
     attn_avg_ms = sum(attn_ms) / len(attn_ms)
     flops_launch = flops_step / wl.num_parts          # zigzag partitions carry equal pair counts
     attn_tflops = flops_launch / (attn_avg_ms * 1e-3) / 1e12
-    items = wl.seq_len * wl.hq
-    merge = None
-    if merge_ms:
-        # Algorithmic bytes of one merge launch over n parts: n reads of (128*4 + 4) B per (row, head) plus one
-        # write (fp32 partial: 516 B; final bf16 output + LSE: 260 B).  Rows of a part with no visible key are
-        # skipped by the kernels, so this is an upper bound on the traffic.
-        per_step = len(runner.merge_parts)
-        out_final = 128 * (2 if wl.dtype == torch.bfloat16 else 4) + 4
-        byts = [items * (n * 516 + (out_final if i == per_step - 1 else 516)) for i, n in enumerate(runner.merge_parts)]
-        total_bytes = sum(byts) * args.steps
-        gbs = total_bytes / (sum(merge_ms) * 1e-3) / 1e9
-        merge = {"launches_per_step": per_step, "parts_per_launch": runner.merge_parts,
-                 "ms_per_launch": sum(merge_ms) / len(merge_ms), "algorithmic_gbs": gbs,
-                 "frac_of_measured_hbm": gbs / peaks["hbm"], "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
-                 "note": "bytes are an upper bound: rows of a part with no visible key are not read"}
     h2d = q_h.numel() * q_h.element_size() + 2 * k_h.numel() * k_h.element_size()
     d2h = o_h.numel() * o_h.element_size() + l_h.numel() * 4
+    del runner, pipe, q, k, v, o_h, l_h
+    torch.cuda.empty_cache()
+
+    # Which measured cuBLAS rate the attention kernel is held against follows from the run itself: a timed
+    # region of seconds sits at the power cap like the sustained GEMM loop, a shorter one runs at burst clocks.
+    timed_s = total_ms * 1e-3
+    kind = "sustained" if timed_s >= 2.0 else "burst"
+    peak = peaks["bf16_sustained"] if kind == "sustained" else peaks["bf16_burst"]
+    counters = stored_counters(wl.name)
+    traffic = None if (counters is None or counters["stale"]) else counters["dram_bytes_per_launch"]
+    sm_mhz = (clocks or {}).get("sm_mhz")
+    roofline = {"bound": "tensor", "kernel": "attn_prefill_bf16_kernel", "achieved": attn_tflops, "peak": peak,
+                "unit": "TFLOP/s", "frac": attn_tflops / peak, "traffic": traffic,
+                "traffic_unit": "bytes per launch (ncu dram read + write, captured offline)",
+                "peak_source": f"{peaks['source']} cuBLAS bf16, {kind} figure (timed region {timed_s:.2f} s)",
+                "frac_of_sustained": attn_tflops / peaks["bf16_sustained"], "frac_of_burst": attn_tflops / peaks["bf16_burst"],
+                "frac_of_nominal": attn_tflops / NOMINAL_BF16_TFLOPS,
+                "flops_per_launch": flops_launch, "ms_per_launch": attn_avg_ms,
+                "ms_per_launch_x_sm_mhz": attn_avg_ms * sm_mhz if sm_mhz else None,
+                "launches_timed": len(attn_ms), "ncu": counters}
+
+    extra = None
+    if world == 1 and not args.no_extra:
+        extra = {}
+        for name, fn in (("c3", extra_partitioned), ("c3_merge_kernel", extra_merge_kernel), ("c4", run_preempted),
+                         ("c2", run_short_batch), ("ring", run_ring), ("decode", run_decode), ("linear", run_linear)):
+            try:
+                extra[name] = fn(args)
+            except Exception as exc:                       # an extra record must not take the headline with it
+                extra[name] = {"error": f"{type(exc).__name__}: {exc}"}
+            torch.cuda.empty_cache()
 
     cpu = oracle_sample(wl, q_h, k_h, v_h, target_s=15.0)
     line = {
@@ -314,14 +352,7 @@ def run_ours(args, wl):
         "frac_of_nominal_bf16_peak": tflops / world / NOMINAL_BF16_TFLOPS,
         "frac_of_measured_bf16_sustained": tflops / world / peaks["bf16_sustained"],
         "attention_only_tflops": attn_tflops,
-        "merge": merge,
-        "roofline": {"bound": "tensor", "kernel": "attn_prefill_bf16_kernel", "achieved": attn_tflops,
-                     "peak": peaks["bf16_sustained"], "unit": "TFLOP/s", "frac": attn_tflops / peaks["bf16_sustained"],
-                     "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "traffic_unit": "bytes per launch (ncu dram read + write)",
-                     "ncu": NCU_PIPES.get(wl.name),
-                     "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside a long step)",
-                     "frac_of_burst": attn_tflops / peaks["bf16_burst"], "frac_of_nominal": attn_tflops / NOMINAL_BF16_TFLOPS,
-                     "flops_per_launch": flops_launch, "ms_per_launch": attn_avg_ms},
+        "roofline": roofline,
         "cpu_baseline": {"value": cpu["tflops"], "unit": "TFLOP/s", "cores": cpu["cores"], "kind": "oracle",
                          "sample": f"{cpu['rows']} seeded random query rows x {wl.hq} heads of the same request, "
                                    f"{cpu['seconds']:.1f} s; tokens/s extrapolated by pair count: "
@@ -331,12 +362,107 @@ def run_ours(args, wl):
                 "how": "consecutive steps pipelined on three streams: every step's H2D, compute and D2H are inside the "
                        "timed region; copies of neighbouring steps overlap the compute",
                 "one_step_at_a_time": {"value": whole_job_tflops(flops_step, world, serial_ms), "ms_per_step": serial_ms}},
-        "gpu_launches": args.steps * runner.launches_per_step(),
+        "gpu_launches": args.steps * launches_per_step,
         "clocks": clocks,
+        "extra": extra,
     }
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def _extra_steps(args, cap):
+    return max(3, min(args.steps, cap))
+
+
+def extra_partitioned(args, name="c3"):
+    """Extra record: the whole partitioned step of another long configuration (every partition's launch merging
+    into the running state), a few steps, with the attention launches timed one by one."""
+    from paper_2409_15104_b200 import binding
+    from paper_2409_15104_b200.prefill import PartitionedPrefill
+    wl = workloads.WORKLOADS[name]
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    q, k, v = (t.to(dev) for t in workloads.qkv(wl.seed, wl.seq_len, wl.hq, wl.hkv, 128, wl.dtype))
+    runner = PartitionedPrefill(wl.seq_len, wl.hq, wl.num_parts, wl.dtype, dev, wl.part_align)
+    for _ in range(max(args.warmup, 3)):
+        runner.run(q, k, v)
+    torch.cuda.synchronize()
+    steps = _extra_steps(args, 20)
+    sampler = ClockSampler(0); sampler.start(); time.sleep(0.2)
+    runner.attn_events = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        runner.run(q, k, v, time_kernels=True)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    binding.check_status()
+    ms = e0.elapsed_time(e1) / steps
+    attn_ms = [a.elapsed_time(b) for a, b in runner.attn_events]
+    fl = workloads.attention_flops(workloads.causal_pairs(wl.seq_len), wl.hq)
+    peaks = load_peaks()
+    attn_tf = fl / wl.num_parts / (sum(attn_ms) / len(attn_ms) * 1e-3) / 1e12
+    counters = stored_counters(wl.name)
+    return {"metric": "whole partitioned step, TFLOP/s (extra record)", "value": fl / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+            "ms_per_step": ms, "steps": steps, "tokens_per_s": wl.seq_len / (ms * 1e-3),
+            "attention_only_tflops": attn_tf, "attention_ms_per_launch": sum(attn_ms) / len(attn_ms),
+            "frac_of_burst": attn_tf / peaks["bf16_burst"], "frac_of_sustained": attn_tf / peaks["bf16_sustained"],
+            "frac_of_nominal": attn_tf / NOMINAL_BF16_TFLOPS,
+            "traffic": None if (counters is None or counters["stale"]) else counters["dram_bytes_per_launch"], "ncu": counters,
+            "launches_per_step": runner.launches_per_step(), "clocks": clocks, "config": workload_config(wl)}
+
+
+def merge_bytes_exact(seq_len, hq, bounds, parts, final_bf16):
+    """DRAM bytes one n-way merge launch must move: part p holds keys from bounds[p] on, so under the causal
+    mask its rows below bounds[p] are empty and the kernel reads only their LSE; every other (row, head) of a
+    part costs 128 fp32 + the LSE, and every (row, head) is written once."""
+    total = 0
+    for p in parts:
+        live = seq_len - bounds[p]
+        total += hq * (live * 516 + (seq_len - live) * 4)
+    total += seq_len * hq * ((256 if final_bf16 else 512) + 4)
+    return total
+
+
+def extra_merge_kernel(args, name="c3"):
+    """Extra record: the n-way LSE merge kernel alone (the path two GPUs' partial outputs take), on the fp32
+    partials of every zigzag partition of c3, HBM-bound, with the exact byte count from the plan."""
+    from paper_2409_15104_b200 import binding
+    wl = workloads.WORKLOADS[name]
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    q, k, v = (t.to(dev) for t in workloads.qkv(wl.seed, wl.seq_len, wl.hq, wl.hkv, 128, wl.dtype))
+    P, S = wl.num_parts, wl.seq_len
+    parts = [binding.pec_prefill_attn(q, k, v, part_id=p, num_parts=P, part_align=wl.part_align) for p in range(P)]
+    out_o = torch.empty((S, wl.hq, 128), dtype=wl.dtype, device=dev)
+    out_l = torch.empty((S, wl.hq), dtype=torch.float32, device=dev)
+    o_parts, l_parts = [x[0] for x in parts], [x[1] for x in parts]
+    for _ in range(3):
+        binding.pec_attn_merge_n(o_parts, l_parts, o_out=out_o, lse_out=out_l)
+    torch.cuda.synchronize()
+    steps = _extra_steps(args, 20)
+    evs = []
+    for _ in range(steps):                                   # 4.3 GB of partials: far beyond the L2
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); binding.pec_attn_merge_n(o_parts, l_parts, o_out=out_o, lse_out=out_l); e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    binding.check_status()
+    ms = statistics.median(a.elapsed_time(b) for a, b in evs)
+    bounds = binding.pec_plan_partitions(S, P, 0, wl.part_align, 128, 128, True, tiles=False)["bounds"]
+    byts = merge_bytes_exact(S, wl.hq, bounds, range(P), wl.dtype == torch.bfloat16)
+    gbs = byts / (ms * 1e-3) / 1e9
+    peaks = load_peaks()
+    return {"metric": "n-way LSE merge kernel, achieved HBM GB/s (extra record)", "value": gbs, "unit": "GB/s", "ms_per_launch": ms,
+            "steps": steps, "parts": P,
+            "roofline": {"bound": "hbm", "kernel": "merge_n_kernel", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
+                         "frac": gbs / peaks["hbm"], "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "traffic": None,
+                         "algorithmic_bytes": byts, "peak_source": peaks["source"] + " copy bandwidth",
+                         "bytes": "exact: rows of a part below its first key are empty and only their LSE is read"},
+            "config": {"workload": f"{wl.name}: {P}-way merge of the partitions' fp32 partials into the bf16 output",
+                       "l2": "partials (4.3 GB) exceed the L2"}}
 
 
 def run_decode(args):
@@ -357,7 +483,7 @@ def run_decode(args):
     for _ in range(max(args.warmup, 3)):
         binding.pec_decode_attn(q, k, v, o=o, lse=lse, workspace=ws)
     torch.cuda.synchronize()
-    steps = min(args.steps, 50)
+    steps = _extra_steps(args, 50)
     evs = []
     for _ in range(steps):
         flush.zero_()
@@ -373,14 +499,14 @@ def run_decode(args):
     import oracle
     want = oracle.attn_rows(q.cpu()[None], [L - 1], k.cpu(), v.cpu(), [(0, L)], False)
     err = float(np.abs(o.float().cpu().double().numpy() - want[0][0]).max())
-    print(json.dumps({"metric": "split-KV decode attention, achieved HBM GB/s (extra line, not the headline)",
+    return {"metric": "split-KV decode attention, achieved HBM GB/s (extra line, not the headline)",
                       "value": gbs, "unit": "GB/s", "ms_per_step": ms, "steps": steps, "n_gpus": 1, "dtype": "bf16",
                       "data": "synthetic", "config": {"workload": f"decode: one token, {hq}/{hkv} heads, {L} cached keys",
                                                        "l2": "256 MiB written between timed calls"},
                       "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
                                    "frac": gbs / peaks["hbm"], "traffic": None,
                                    "algorithmic_bytes": byts, "peak_source": peaks["source"] + " copy bandwidth"},
-                      "max_abs_err_vs_oracle": err}), flush=True)
+                      "max_abs_err_vs_oracle": err}
 
 
 def run_linear(args):
@@ -396,7 +522,7 @@ def run_linear(args):
     for _ in range(max(args.warmup, 3)):
         binding.pec_linear(x, w, y=y)
     torch.cuda.synchronize()
-    steps = min(args.steps, 50)
+    steps = _extra_steps(args, 50)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(steps):
@@ -411,13 +537,13 @@ def run_linear(args):
     rows = [0, 1, 127, 128, 4095, M - 1]
     want = oracle.linear(x[rows].cpu(), w.cpu())
     err = float(np.abs(y[rows].float().cpu().double().numpy() - want).max())
-    print(json.dumps({"metric": "QKV-generation GEMM TFLOP/s (extra line, not the headline)", "value": tf, "unit": "TFLOP/s",
+    return {"metric": "QKV-generation GEMM TFLOP/s (extra line, not the headline)", "value": tf, "unit": "TFLOP/s",
                       "ms_per_step": ms, "steps": steps, "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
                       "config": {"workload": f"linear: x [{M},{K}] times w [{N},{K}]^T", "l2": "operands and output (752 MB) exceed L2"},
                       "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
                                    "frac": tf / peaks["bf16_sustained"], "traffic": None,
                                    "peak_source": peaks["source"] + " sustained cuBLAS bf16"},
-                      "max_abs_err_vs_oracle_sampled_rows": err}), flush=True)
+                      "max_abs_err_vs_oracle_sampled_rows": err}
 
 
 def _short_batch(wl, dev, seed_offset=0):
@@ -443,7 +569,7 @@ def run_ring(args):
         _, _, launches = ring_prefill(q, k, v, P, wl.part_align)
     torch.cuda.synchronize()
     evs = []
-    for _ in range(min(args.steps, 20)):
+    for _ in range(_extra_steps(args, 20)):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(); ring_prefill(q, k, v, P, wl.part_align); e1.record()
         evs.append((e0, e1))
@@ -454,141 +580,182 @@ def run_ring(args):
     plans = {name: binding.pec_plan_ring(wl.seq_len, P, wl.part_align, code, True)
              for name, code in (("zigzag", binding.PEC_LAYOUT_ZIGZAG), ("contiguous", binding.PEC_LAYOUT_CONTIGUOUS))}
     total = workloads.causal_pairs(wl.seq_len)
-    print(json.dumps({"metric": "ring-attention SP steps of all ranks on one GPU, attention TFLOP/s (extra line, not the headline)",
+    return {"metric": "ring-attention SP steps of all ranks on one GPU, attention TFLOP/s (extra line, not the headline)",
                       "value": fl / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms, "n_gpus": 1, "dtype": "bf16",
                       "data": "synthetic", "gpu_launches_per_step": launches,
                       "planned_ring_time_in_pairs": {name: sum(pl["step_max"]) for name, pl in plans.items()},
                       "planned_ring_efficiency": {name: total / (P * sum(pl["step_max"])) for name, pl in plans.items()},
                       "config": {"workload": f"ring: {wl.note}; rank r's query blocks against the keys of rank (r-t) mod P",
-                                 "ranks": P, "l2": "inputs and partials exceed the 126 MB L2"}}), flush=True)
+                                 "ranks": P, "l2": "inputs and partials exceed the 126 MB L2"}}
 
 
-def run_short_batch(args, wl):
-    """Extra line: the packed short-request batch (c2) alone."""
+def run_short_batch(args, wl=None):
+    """Extra record: the packed short-request batch (c2) alone.  A step is what a caller does per batch: build
+    the heaviest-first work-list on the host, copy it to the device, launch.  The same batch with every CTA
+    searching cu_seqlens instead is timed beside it."""
     from paper_2409_15104_b200 import binding
-    from paper_2409_15104_b200.prefill import varlen_prefill
+    from paper_2409_15104_b200.prefill import make_worklist, varlen_prefill
+    wl = wl or workloads.WORKLOADS["c2"]
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     q, k, v, cu, T, pairs = _short_batch(wl, dev)
+    cu_host = [int(x) for x in cu.cpu()]
     o = torch.empty((T, wl.hq, 128), dtype=wl.dtype, device=dev)
     lse = torch.empty((T, wl.hq), dtype=torch.float32, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    for _ in range(max(args.warmup, 3)):
+
+    def with_list():
+        varlen_prefill(q, k, v, cu, o=o, lse=lse, worklist=make_worklist(cu_host, wl.dtype, dev))
+
+    def without():
         varlen_prefill(q, k, v, cu, o=o, lse=lse)
-    torch.cuda.synchronize()
-    evs = []
-    for _ in range(min(args.steps, 50)):
-        flush.zero_()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(); varlen_prefill(q, k, v, cu, o=o, lse=lse); e1.record()
-        evs.append((e0, e1))
-    torch.cuda.synchronize()
-    binding.check_status()
-    ms = statistics.median(a.elapsed_time(b) for a, b in evs)
+
+    res = {}
+    for name, fn in (("worklist", with_list), ("search", without)):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        evs = []
+        for _ in range(_extra_steps(args, 50)):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        binding.check_status()
+        res[name] = statistics.median(a.elapsed_time(b) for a, b in evs)
+    ms = res["worklist"]
     fl = workloads.attention_flops(pairs, wl.hq)
-    print(json.dumps({"metric": "short-request varlen batch, attention TFLOP/s (extra line, not the headline)",
-                      "value": fl / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms, "n_gpus": 1, "dtype": "bf16",
-                      "data": "synthetic", "tokens_per_s": T / (ms * 1e-3),
-                      "config": {"workload": f"{wl.name}: {wl.note}", "requests": wl.short_batch, "tokens": T,
-                                 "pairs_per_head": pairs, "l2": "256 MiB written between timed calls"}}), flush=True)
+    peaks = load_peaks()
+    tf = fl / (ms * 1e-3) / 1e12
+    return {"metric": "short-request varlen batch, attention TFLOP/s (extra record)",
+            "value": tf, "unit": "TFLOP/s", "ms_per_step": ms, "n_gpus": 1, "dtype": "bf16",
+            "data": "synthetic", "tokens_per_s": T / (ms * 1e-3),
+            "frac_of_burst": tf / peaks["bf16_burst"], "frac_of_nominal": tf / NOMINAL_BF16_TFLOPS,
+            "without_worklist": {"value": fl / (res["search"] * 1e-3) / 1e12, "ms_per_step": res["search"]},
+            "config": {"workload": f"{wl.name}: {wl.note}", "requests": wl.short_batch, "tokens": T,
+                       "pairs_per_head": pairs, "l2": "256 MiB written between timed calls"}}
 
 
-def run_preempted(args, wl):
-    """Extra line: c4 - a long prefill as 16 resumed chunks on a low-priority stream with a short-request
-    batch arriving on a high-priority stream while chunk 4 runs."""
+def run_preempted(args, wl=None):
+    """Extra record: c4 - a long prefill as 16 resumed chunks on a low-priority stream with a short-request
+    batch on a high-priority stream, arriving (a) at a chunk boundary and (b) in the middle of a late chunk,
+    which is what preemption between kernels costs a short request: the rest of the running chunk at worst."""
     from paper_2409_15104_b200 import binding
-    from paper_2409_15104_b200.prefill import chunked_prefill, varlen_prefill
+    from paper_2409_15104_b200.prefill import chunked_prefill, make_worklist, varlen_prefill
+    wl = wl or workloads.WORKLOADS["c4"]
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     S, C = wl.seq_len, wl.chunk_len
     q, k, v = (t.to(dev) for t in workloads.qkv(wl.seed, S, wl.hq, wl.hkv, 128, wl.dtype))
     sq, sk, sv, cu, T, spairs = _short_batch(wl, dev)
+    slist = make_worklist([int(x) for x in cu.cpu()], wl.dtype, dev)
     o = torch.empty((S, wl.hq, 128), dtype=wl.dtype, device=dev)
     lse = torch.empty((S, wl.hq), dtype=torch.float32, device=dev)
     so = torch.empty((T, wl.hq, 128), dtype=wl.dtype, device=dev)
     sl = torch.empty((T, wl.hq), dtype=torch.float32, device=dev)
     lo, hi = torch.cuda.Stream(priority=0), torch.cuda.Stream(priority=-1)
+    n_chunks = S // C
+    late = n_chunks - 4                                       # the chunk the batch interrupts in (b)
 
     def timed(fn):
         torch.cuda.synchronize()
         t0 = time.perf_counter(); fn(); torch.cuda.synchronize()
         return (time.perf_counter() - t0) * 1e3
 
-    def long_only():
-        chunked_prefill(q, k, v, C, o, lse, stream=lo)
+    def long_only(events=None):
+        chunked_prefill(q, k, v, C, o, lse, stream=lo, events=events)
 
     def short_only():
-        varlen_prefill(sq, sk, sv, cu, o=so, lse=sl, stream=hi)
+        varlen_prefill(sq, sk, sv, cu, o=so, lse=sl, stream=hi, worklist=slist)
 
     marks = {}
 
-    def both():
+    def short_timed(key):
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(hi); short_only(); s1.record(hi)
+        marks[key] = (s0, s1)
+
+    def at_boundary():
         def arrive(c):
-            if c == 3:                                         # the batch arrives once chunk 3 has finished
-                ev = torch.cuda.Event(enable_timing=True); ev.record(lo)
+            if c == 3:                                         # the batch starts once chunk 3 has finished
+                ev = torch.cuda.Event(); ev.record(lo)
                 hi.wait_event(ev)
-                s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                s0.record(hi); short_only(); s1.record(hi)
-                marks["short"] = (s0, s1)
+                short_timed("boundary")
         chunked_prefill(q, k, v, C, o, lse, stream=lo, between_chunks=arrive)
 
-    for fn in (long_only, short_only, both):
+    def mid_chunk():
+        started = {}
+
+        def arrive(c):
+            if c == late - 1:
+                started["ev"] = torch.cuda.Event(); started["ev"].record(lo)
+            if c == n_chunks - 1:                              # every chunk is enqueued: now wait, on the host, for chunk
+                started["ev"].synchronize()                    # `late` to be the one running, let it run for a while,
+                time.sleep(0.003)                              # and only then hand the batch to the GPU
+                short_timed("mid")
+        chunked_prefill(q, k, v, C, o, lse, stream=lo, between_chunks=arrive)
+
+    for fn in (long_only, short_only, at_boundary, mid_chunk):
         timed(fn)                                              # warm-up
     reps = 3
-    t_long = min(timed(long_only) for _ in range(reps))
+    chunk_events = []
+    t_long = min(timed(lambda: long_only(chunk_events)) for _ in range(reps))
+    chunk_ms = [a.elapsed_time(b) for a, b in chunk_events]
     t_short = min(timed(short_only) for _ in range(reps))
-    t_both, lat = [], []
+    t_both, lat_b, lat_m = [], [], []
     for _ in range(reps):
-        t_both.append(timed(both))
-        lat.append(marks["short"][0].elapsed_time(marks["short"][1]))
+        t_both.append(timed(at_boundary))
+        lat_b.append(marks["boundary"][0].elapsed_time(marks["boundary"][1]))
+        timed(mid_chunk)
+        lat_m.append(marks["mid"][0].elapsed_time(marks["mid"][1]))
     binding.check_status()
     fl_long = workloads.attention_flops(workloads.causal_pairs(S), wl.hq)
     fl_short = workloads.attention_flops(spairs, wl.hq)
-    print(json.dumps({"metric": "preempted long prefill with a colocated short batch (extra line, not the headline)",
-                      "value": (fl_long + fl_short) / (min(t_both) * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": 1,
-                      "dtype": "bf16", "data": "synthetic",
-                      "long_alone_ms": t_long, "long_alone_tflops": fl_long / (t_long * 1e-3) / 1e12,
-                      "short_alone_ms": t_short, "interleaved_ms": min(t_both),
-                      "short_batch_latency_when_colocated_ms": min(lat), "short_batch_latency_worst_ms": max(lat),
-                      "timing": "host wall clock around a synchronised region (multi-stream); short latency by CUDA events",
-                      "config": {"workload": f"{wl.name}: {wl.note}", "chunks": S // C, "short_tokens": T}}), flush=True)
+    peaks = load_peaks()
+    tf_long = fl_long / (t_long * 1e-3) / 1e12
+    return {"metric": "preempted long prefill with a colocated short batch (extra record)",
+            "value": (fl_long + fl_short) / (min(t_both) * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": 1,
+            "dtype": "bf16", "data": "synthetic",
+            "long_alone_ms": t_long, "long_alone_tflops": tf_long, "long_alone_frac_of_nominal": tf_long / NOMINAL_BF16_TFLOPS,
+            "long_alone_frac_of_sustained": tf_long / peaks["bf16_sustained"], "long_tokens_per_s": S / (t_long * 1e-3),
+            "short_alone_ms": t_short, "interleaved_ms": min(t_both),
+            "short_batch_latency_at_chunk_boundary_ms": {"best": min(lat_b), "worst": max(lat_b)},
+            "short_batch_latency_arriving_mid_chunk_ms": {"best": min(lat_m), "worst": max(lat_m), "interrupted_chunk": late,
+                                                          "that_chunk_alone_ms": chunk_ms[late] if len(chunk_ms) > late else None},
+            "longest_chunk_ms": max(chunk_ms) if chunk_ms else None,
+            "timing": "host wall clock around a synchronised region (multi-stream); short-batch latency by CUDA events on its "
+                      "own stream, from the moment the host hands it over to its completion",
+            "config": {"workload": f"{wl.name}: {wl.note}", "chunks": n_chunks, "short_tokens": T}}
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode", "linear", "ring"], default="c3")
+    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode", "linear", "ring", "merge"], default="c5",
+                    help="c5 (default, the largest single-GPU configuration) and c3 print the full line; the others "
+                         "print their extra record alone")
+    ap.add_argument("--no-extra", action="store_true", help="skip the extra records nested under the headline line")
     ap.add_argument("--reference-seconds", type=float, default=0.0,
                     help="--impl reference: CPU seconds per step (default: 90 s spread over the steps, 0.15-20 s each)")
     ap.add_argument("--profile", action="store_true",
-                    help="profiling runs: skip the end-to-end and CPU-baseline legs (the printed line is not a result)")
+                    help="profiling runs: skip the end-to-end, extra and CPU-baseline legs (the printed line is not a result)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.workload == "decode":
-        run_decode(args)
-        return
-    if args.workload == "linear":
-        run_linear(args)
-        return
-    if args.workload == "ring":
-        run_ring(args)
-        return
-    wl = workloads.WORKLOADS[args.workload]
-    if args.workload == "c2":
-        run_short_batch(args, wl)
-        return
-    if args.workload == "c4":
-        run_preempted(args, wl)
-        return
     if args.impl == "reference":
-        run_reference(args, wl)
-    else:
-        if not torch.cuda.is_available():
-            raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
-        run_ours(args, wl)
+        run_reference(args, workloads.WORKLOADS[args.workload if args.workload in ("c3", "c5") else "c5"])
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
+    alone = {"decode": run_decode, "linear": run_linear, "ring": run_ring, "c2": run_short_batch, "c4": run_preempted,
+             "merge": extra_merge_kernel}
+    if args.workload in alone:
+        print(json.dumps(alone[args.workload](args)), flush=True)
+        return
+    run_ours(args, workloads.WORKLOADS[args.workload])
 
 
 if __name__ == "__main__":

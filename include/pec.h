@@ -66,6 +66,12 @@ enum { PEC_TILE_SKIP = 0, PEC_TILE_PARTIAL = 1, PEC_TILE_FULL = 2 };
  * chunk_start must be 0, chunk_len and kv_len must equal seq_len, num_parts
  * must be 1.
  *
+ * Query subset: with q_num_parts <= 1 every row of the chunk; otherwise only those rows of the
+ * chunk that lie in zigzag partition q_part_id of q_num_parts (same rule and part_align as the key
+ * partitions): the rows one rank of ring-attention sequence parallelism keeps (Section 2.2), so that
+ * one call with part_id = (q_part_id - t) mod num_parts is that rank's ring step t.  o and lse keep
+ * their chunk layout; rows outside the query subset are neither read nor written.  Single request only.
+ *
  * Key subset: with num_parts == 1 all keys of [0, kv_len); otherwise zigzag
  * partition part_id of num_parts as defined by pec_plan_partitions(seq_len,
  * num_parts, ..., part_align, ...), intersected with [0, kv_len).  With
@@ -77,6 +83,18 @@ enum { PEC_TILE_SKIP = 0, PEC_TILE_PARTIAL = 1, PEC_TILE_FULL = 2 };
  * with no visible key gets o = 0 and lse = -inf, the identity of
  * pec_attn_merge.  o_dtype PEC_F32 gives a partial fit for merging;
  * PEC_BF16 rounds to nearest-even (allowed with in_dtype PEC_BF16 only).
+ *
+ * Incoming state (acc_o, acc_lse; both or neither): a partial result of the SAME rows over a key
+ * subset disjoint from this call's, fp32, laid out like o / lse.  The call then returns the merge of
+ * the two - lse = ln(exp(acc_lse) + exp(lse_own)), o = the correspondingly weighted sum, i.e. the
+ * online-softmax step across key segments of Section 2.2, what pec_attn_merge computes - instead of
+ * its own partial, so a chain of calls over the key partitions needs no partial buffers and no merge
+ * pass.  o / lse may be the very buffers acc_o / acc_lse (both, o_dtype PEC_F32): rows that see no key
+ * of this call's subset then stay untouched.  Only the last call of a chain should round to PEC_BF16.
+ *
+ * Packed batches may pass a work-list (worklist, n_items, worklist_block_m) made by pec_plan_worklist
+ * and copied to the device by the caller: tiles then run heaviest first across requests and no CTA
+ * searches cu_seqlens.  worklist_block_m must equal pec_worklist_block_m(in_dtype).
  *
  * in_dtype PEC_BF16 runs the tcgen05 tensor-core kernel (bf16 products, fp32
  * accumulation); PEC_F32 runs an fp32 FMA kernel (accuracy path).
@@ -102,13 +120,22 @@ typedef struct {
     float softmax_scale;        /* 0 selects 1/sqrt(D)                                   */
     void *workspace;            /* device scratch of pec_workspace_size() bytes or NULL  */
     size_t workspace_bytes;
-    int32_t *status;            /* device word, may be NULL; the caller zeroes it; a     */
-                                /* kernel stores PEC_ERR_TIMEOUT there if a wait expired */
+    int32_t *status;            /* device word the caller zeroes; a kernel stores        */
+                                /* PEC_ERR_TIMEOUT there if a wait expired.  Required    */
+                                /* for in_dtype PEC_BF16, may be NULL for PEC_F32        */
+    const float *acc_o;         /* device; incoming state [rows, Hq, D] fp32, or NULL    */
+    const float *acc_lse;       /* device; [rows, Hq] fp32, or NULL                      */
+    int32_t q_part_id, q_num_parts;   /* q_num_parts <= 1: all rows of the chunk         */
+    const int32_t *worklist;    /* device; [n_items][4] from pec_plan_worklist, or NULL  */
+    int32_t n_items;
+    int32_t worklist_block_m;
 } pec_attn_args;
 
 /*
  * Partial attention of one chunk / partition / packed batch (Eq. 3-4; see the
- * struct above).  Validates the arguments on the host, then enqueues one kernel.
+ * struct above).  Validates the arguments on the host, then enqueues the attention
+ * kernel over the row tiles that can see a key of the subset and, where whole tiles
+ * of rows see none and still have to be written, one small fill kernel for those.
  * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.
  */
 int pec_prefill_attn(const pec_attn_args *args, void *cuda_stream);
@@ -209,7 +236,11 @@ size_t pec_decode_workspace_size(const pec_decode_args *args);
  * names both sizes: lower num_splits, or use pec_decode_attn.
  *
  * The first call on each device looks up the array's device address (with that device
- * current) and remembers it; make that first call outside any stream capture.  All calls on a
+ * current) and remembers it; make that first call outside any stream capture.  Under CUDA's
+ * default lazy module loading that first call may also be the moment the driver loads the part
+ * of the library that holds the array, i.e. the moment the array's memory is actually taken: an
+ * engine should therefore make one priming call per device at start-up, before it sizes its
+ * pool (or run with CUDA_MODULE_LOADING=EAGER).  Every later call takes and returns no memory.  All calls on a
  * device share the one array and it keeps whatever the previous call left there.  Nothing in
  * it has to start at zero - each call overwrites every partial it later reads - but two calls
  * that overlap on the GPU (different streams, or one stream replayed concurrently) would
@@ -250,6 +281,25 @@ typedef struct {
 /* Errors: INVALID_ARG (seq_len < 0, num_parts < 1, align/block < 1, NULL plan), CAPACITY. */
 int pec_plan_partitions(int64_t seq_len, int32_t num_parts, int64_t chunk_len, int32_t align,
                         int32_t block_m, int32_t block_n, int32_t causal, pec_plan *plan);
+
+/*
+ * Work-list of a packed batch of short requests (Section 5.2): one entry per tile of block_m query
+ * rows, every request starting a fresh tile, ordered so that the kernel's CTAs take the tiles with
+ * the most key tiles first (a heavy tile started late would leave the other SMs idle at the end).
+ *   weight of the tile at positions [pos0, pos0 + n) of a request of length L:
+ *       causal: ceil(min(L, pos0 + n) / block_n), otherwise ceil(L / block_n)
+ *   order: weight descending; equal weights by request index, then pos0, ascending
+ *   items[4 i .. 4 i + 3] = { cu_seqlens[b], pos0, n, L } of entry i (request b)
+ * cu_seqlens: HOST [B + 1], non-decreasing, starting anywhere; items: HOST, capacity items_cap entries
+ * (may be NULL for a size query); *n_items receives the number of entries, sum_b ceil(L_b / block_m).
+ * The caller copies items to the device and passes it as pec_attn_args.worklist.
+ * Errors: INVALID_ARG (NULL cu_seqlens or n_items, B < 0, decreasing offsets, block < 1), CAPACITY.
+ */
+int pec_plan_worklist(const int32_t *cu_seqlens, int32_t B, int32_t block_m, int32_t block_n, int32_t causal,
+                      int32_t *items, int64_t items_cap, int64_t *n_items);
+
+/* Query rows per tile of the kernel behind pec_prefill_attn for this input type (0: unknown type). */
+int32_t pec_worklist_block_m(int32_t in_dtype);
 
 /*
  * Work plan of ring-attention sequence parallelism over num_parts ranks (Section 2.2: each replica
@@ -327,6 +377,24 @@ int pec_select_sp(const pec_sp_inputs *in, pec_sp_choice *out);
  */
 int pec_linear(const void *x, int64_t x_stride, const void *w, int64_t w_stride, void *y, int64_t y_stride,
                int64_t M, int32_t N, int32_t K, int32_t *status, void *cuda_stream);
+
+/*
+ * Process-wide settings (the paper has no counterpart; they exist for operations and tests).
+ *   PEC_CTL_WAIT_LIMIT_CYCLES   limit of every barrier wait inside the kernels, in SM clock cycles
+ *                               (default 2e9, about a second).  A wait that runs out makes its CTA
+ *                               leave through the normal exit and stores PEC_ERR_TIMEOUT in the
+ *                               status word; a serving engine that would rather lose a request than
+ *                               stall every short request queued behind a stuck kernel (Section 5.1's
+ *                               preemption works between kernels only) sets it lower.  value >= 1000.
+ *   PEC_CTL_TEST_SKIP_LAST_LOAD test hook, 0 / 1: the loader of the tensor-core kernels leaves out its
+ *                               last tile (attention: the last V tile of a CTA that walks at least two
+ *                               key tiles; pec_linear: the last K step of the second CTA of each pair),
+ *                               so that the waits for it run out and the timeout path can be checked.
+ *                               Results of such a launch are undefined; the status word tells.
+ * Applies to launches enqueued after the call.  Errors: INVALID_ARG.
+ */
+enum { PEC_CTL_WAIT_LIMIT_CYCLES = 1, PEC_CTL_TEST_SKIP_LAST_LOAD = 2 };
+int pec_control(int32_t what, int64_t value);
 
 /* Text describing the last non-zero return on this thread (never NULL). */
 const char *pec_last_error(void);

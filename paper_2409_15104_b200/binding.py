@@ -46,6 +46,9 @@ class pec_attn_args(ctypes.Structure):
         ("softmax_scale", ctypes.c_float),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("status", ctypes.c_void_p),
+        ("acc_o", ctypes.c_void_p), ("acc_lse", ctypes.c_void_p),
+        ("q_part_id", ctypes.c_int32), ("q_num_parts", ctypes.c_int32),
+        ("worklist", ctypes.c_void_p), ("n_items", ctypes.c_int32), ("worklist_block_m", ctypes.c_int32),
     ]
 
 
@@ -89,7 +92,8 @@ class pec_plan(ctypes.Structure):
 
 EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_attn_merge_n", "pec_plan_partitions",
            "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size", "pec_decode_attn_static", "pec_select_sp", "pec_linear",
-           "pec_plan_ring", "pec_balance_batches")
+           "pec_plan_ring", "pec_balance_batches", "pec_plan_worklist", "pec_worklist_block_m", "pec_control")
+PEC_CTL_WAIT_LIMIT_CYCLES, PEC_CTL_TEST_SKIP_LAST_LOAD = 1, 2
 PEC_DECODE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 PEC_MERGE_MAX_PARTS = 16
 
@@ -136,6 +140,14 @@ def load():
     lib.pec_balance_batches.restype = ctypes.c_int
     lib.pec_balance_batches.argtypes = [ctypes.POINTER(ctypes.c_int32), ctypes.c_int32, ctypes.c_int32,
                                         ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)]
+    lib.pec_plan_worklist.restype = ctypes.c_int
+    lib.pec_plan_worklist.argtypes = [ctypes.POINTER(ctypes.c_int32), ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                      ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), ctypes.c_int64,
+                                      ctypes.POINTER(ctypes.c_int64)]
+    lib.pec_worklist_block_m.restype = ctypes.c_int32
+    lib.pec_worklist_block_m.argtypes = [ctypes.c_int32]
+    lib.pec_control.restype = ctypes.c_int
+    lib.pec_control.argtypes = [ctypes.c_int32, ctypes.c_int64]
     lib.pec_last_error.restype = ctypes.c_char_p
     lib.pec_last_error.argtypes = []
     _lib = lib
@@ -185,13 +197,18 @@ def check_status(device=None):
 
 def pec_prefill_attn(q, k, v, *, seq_len=None, chunk_start=0, chunk_len=None, kv_len=None,
                      part_id=0, num_parts=1, part_align=128, causal=True, softmax_scale=0.0,
-                     cu_seqlens=None, out_dtype=None, o=None, lse=None, stream=None):
+                     cu_seqlens=None, out_dtype=None, o=None, lse=None, stream=None,
+                     acc=None, q_part_id=0, q_num_parts=0, worklist=None):
     """Partial attention of one chunk / partition / packed batch; returns (o, lse).
 
     q [T, Hq, 128], k / v [Tk, Hkv, 128] CUDA tensors (last dim contiguous).  Single request:
     rows are positions, the call covers query rows [chunk_start, chunk_start+chunk_len) against
     keys [0, kv_len).  Packed batch: pass cu_seqlens (int32 CUDA tensor [B+1]).
     o / lse may be passed in (views are fine as long as they are contiguous).
+    acc = (o, lse) fp32 tensors: an incoming state of the same rows that the call merges its result
+    into (pass the same tensors as o / lse for an in-place chain).  q_num_parts > 1 restricts the
+    query rows to zigzag partition q_part_id.  worklist: int32 CUDA tensor [n, 4] from
+    pec_plan_worklist (packed batches).
     """
     lib = load()
     assert q.is_cuda and k.is_cuda and v.is_cuda
@@ -230,6 +247,16 @@ def pec_prefill_attn(q, k, v, *, seq_len=None, chunk_start=0, chunk_len=None, kv
     a.softmax_scale = float(softmax_scale)
     a.workspace, a.workspace_bytes = None, 0
     a.status = status_word(q.device).data_ptr()
+    if acc is not None:
+        acc_o, acc_l = acc
+        assert acc_o.is_contiguous() and acc_l.is_contiguous() and acc_o.dtype == torch.float32 and acc_l.dtype == torch.float32
+        assert acc_o.shape == (chunk_len, Hq, D) and acc_l.shape == (chunk_len, Hq)
+        a.acc_o, a.acc_lse = acc_o.data_ptr(), acc_l.data_ptr()
+    a.q_part_id, a.q_num_parts = q_part_id, q_num_parts
+    if worklist is not None:
+        assert worklist.is_cuda and worklist.dtype == torch.int32 and worklist.is_contiguous()
+        a.worklist, a.n_items = worklist.data_ptr(), worklist.shape[0]
+        a.worklist_block_m = int(lib.pec_worklist_block_m(a.in_dtype))
     _check(lib.pec_prefill_attn(ctypes.byref(a), _stream_ptr(stream)))
     return o, lse
 
@@ -383,6 +410,29 @@ def pec_plan_partitions(seq_len, num_parts, chunk_len=0, align=128, block_m=128,
         "chunks": [(int(cs[c]), int(cl[c])) for c in range(nch)],
         "nq_tiles": int(plan.nq_tiles), "nk_tiles": int(plan.nk_tiles), "tile_class": tc,
     }
+
+
+def pec_plan_worklist(cu_seqlens, block_m, block_n=128, causal=True):
+    """Heaviest-first tile list of a packed batch (see include/pec.h) as a numpy int32 array [n, 4];
+    cu_seqlens is a host sequence of B + 1 offsets."""
+    import numpy as np
+    lib = load()
+    cu = (ctypes.c_int32 * len(cu_seqlens))(*[int(x) for x in cu_seqlens])
+    B = len(cu_seqlens) - 1
+    n = ctypes.c_int64(0)
+    _check(lib.pec_plan_worklist(cu, B, block_m, block_n, 1 if causal else 0, None, 0, ctypes.byref(n)))
+    items = np.zeros((max(n.value, 1), 4), dtype=np.int32)
+    _check(lib.pec_plan_worklist(cu, B, block_m, block_n, 1 if causal else 0,
+                                 items.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), items.shape[0], ctypes.byref(n)))
+    return items[:n.value]
+
+
+def pec_worklist_block_m(dtype) -> int:
+    return int(load().pec_worklist_block_m(_dtype_code(dtype)))
+
+
+def pec_control(what, value):
+    _check(load().pec_control(what, value))
 
 
 def pec_plan_ring(seq_len, num_parts, align=128, layout=PEC_LAYOUT_ZIGZAG, causal=True):

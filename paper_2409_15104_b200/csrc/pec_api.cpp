@@ -1,8 +1,10 @@
 // C-ABI entry points: argument checks, resolution of the key subset, kernel dispatch.
+#include <atomic>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <climits>
 #include "pec_internal.h"
 
 namespace pec {
@@ -16,6 +18,13 @@ void set_error(const char *fmt, ...)
     vsnprintf(g_last_error, sizeof(g_last_error), fmt, ap);
     va_end(ap);
 }
+
+static std::atomic<int64_t> g_wait_limit_cycles{2000000000LL};   // about a second of SM clock
+static std::atomic<int32_t> g_test_skip_last_load{0};
+int64_t wait_limit_cycles() { return g_wait_limit_cycles.load(std::memory_order_relaxed); }
+int32_t test_skip_last_load() { return g_test_skip_last_load.load(std::memory_order_relaxed); }
+
+constexpr int32_t kBlockMBf16 = 256, kBlockMF32 = 64;   // query rows per CTA of the two attention kernels
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -59,6 +68,33 @@ static int resolve(const pec_attn_args *a, AttnParams &p)
         return PEC_ERR_INVALID_ARG;
     }
     if (!(a->softmax_scale >= 0.f) || std::isinf(a->softmax_scale)) { set_error("pec_prefill_attn: softmax_scale must be finite and >= 0"); return PEC_ERR_INVALID_ARG; }
+    if ((a->acc_o == nullptr) != (a->acc_lse == nullptr)) { set_error("pec_prefill_attn: acc_o and acc_lse go together"); return PEC_ERR_INVALID_ARG; }
+    if (a->acc_o) {
+        const bool alias_o = static_cast<const void *>(a->acc_o) == a->o, alias_l = a->acc_lse == a->lse;
+        if (alias_o != alias_l || (alias_o && a->o_dtype != PEC_F32)) {
+            set_error("pec_prefill_attn: o / lse may be the incoming state's buffers only both at once and with fp32 output");
+            return PEC_ERR_INVALID_ARG;
+        }
+        if (!aligned16(a->acc_o) || (reinterpret_cast<uintptr_t>(a->acc_lse) & 3u)) {
+            set_error("pec_prefill_attn: acc_o must be 16-byte aligned (acc_lse 4-byte)");
+            return PEC_ERR_ALIGNMENT;
+        }
+    }
+    if (a->q_num_parts > 1 && (a->q_part_id < 0 || a->q_part_id >= a->q_num_parts || a->cu_seqlens)) {
+        set_error("pec_prefill_attn: need 0 <= q_part_id < q_num_parts, single request only");
+        return PEC_ERR_INVALID_ARG;
+    }
+    if (a->in_dtype == PEC_BF16 && !a->status) { set_error("pec_prefill_attn: bf16 inputs need a status word"); return PEC_ERR_INVALID_ARG; }
+    if (a->worklist) {
+        if (!a->cu_seqlens || a->n_items < 0 || (reinterpret_cast<uintptr_t>(a->worklist) & 15u)) {
+            set_error("pec_prefill_attn: a work-list needs cu_seqlens, n_items >= 0 and 16-byte alignment");
+            return PEC_ERR_INVALID_ARG;
+        }
+        if (a->worklist_block_m != pec_worklist_block_m(a->in_dtype)) {
+            set_error("pec_prefill_attn: work-list built for tiles of %d rows, this kernel uses %d", a->worklist_block_m, pec_worklist_block_m(a->in_dtype));
+            return PEC_ERR_INVALID_ARG;
+        }
+    }
     if (a->cu_seqlens) {
         if (a->B < 1) { set_error("pec_prefill_attn: packed batch needs B >= 1"); return PEC_ERR_INVALID_ARG; }
         if (a->chunk_start != 0 || a->chunk_len != a->seq_len || a->kv_len != a->seq_len || a->num_parts != 1) {
@@ -89,8 +125,24 @@ static int resolve(const pec_attn_args *a, AttnParams &p)
     p.v_stride_t = a->v_stride_t; p.v_stride_h = a->v_stride_h;
     p.Hq = a->Hq; p.Hkv = a->Hkv; p.group = a->Hq / a->Hkv;
     p.cu_seqlens = a->cu_seqlens; p.B = a->cu_seqlens ? a->B : 1;
-    p.chunk_start = a->chunk_start; p.chunk_len = a->chunk_len;
+    p.worklist = a->worklist; p.n_items = a->worklist ? a->n_items : 0;
     p.total_rows = a->chunk_len;
+    p.out_pos0 = a->chunk_start;
+    p.acc_o = a->acc_o; p.acc_lse = a->acc_lse;
+    p.wait_cycles = wait_limit_cycles();
+    p.test_skip_last_load = test_skip_last_load();
+    // Query rows: the chunk, or its intersection with the two blocks of zigzag partition q_part_id.
+    p.n_qseg = 0;
+    if (!a->cu_seqlens) {
+        int64_t qlo[2] = {a->chunk_start, 0}, qhi[2] = {a->chunk_start + a->chunk_len, 0};
+        int nq = 1;
+        if (a->q_num_parts > 1) { zigzag_intervals(a->seq_len, a->q_num_parts, a->q_part_id, a->part_align, qlo, qhi); nq = 2; }
+        for (int t = 0; t < nq; ++t) {
+            const int64_t lo = qlo[t] > a->chunk_start ? qlo[t] : a->chunk_start;
+            const int64_t hi = qhi[t] < a->chunk_start + a->chunk_len ? qhi[t] : a->chunk_start + a->chunk_len;
+            if (hi > lo) { p.q_lo[p.n_qseg] = lo; p.q_hi[p.n_qseg] = hi; ++p.n_qseg; }
+        }
+    }
     p.causal = a->causal;
     p.scale = a->softmax_scale > 0.f ? a->softmax_scale : (float)(1.0 / std::sqrt((double)kHeadDim));
     p.scale_log2 = (float)((double)p.scale * 1.4426950408889634074);
@@ -120,13 +172,51 @@ extern "C" const char *pec_last_error(void) { return g_last_error; }
 
 extern "C" size_t pec_workspace_size(const pec_attn_args *) { return 0; }
 
+extern "C" int32_t pec_worklist_block_m(int32_t in_dtype)
+{
+    return in_dtype == PEC_BF16 ? kBlockMBf16 : (in_dtype == PEC_F32 ? kBlockMF32 : 0);
+}
+
+extern "C" int pec_control(int32_t what, int64_t value)
+{
+    if (what == PEC_CTL_WAIT_LIMIT_CYCLES && value >= 1000) { g_wait_limit_cycles.store(value); return PEC_OK; }
+    if (what == PEC_CTL_TEST_SKIP_LAST_LOAD && (value == 0 || value == 1)) { g_test_skip_last_load.store((int32_t)value); return PEC_OK; }
+    set_error("pec_control: unknown setting %d or value %lld out of range", (int)what, (long long)value);
+    return PEC_ERR_INVALID_ARG;
+}
+
 extern "C" int pec_prefill_attn(const pec_attn_args *args, void *cuda_stream)
 {
     AttnParams p;
-    const int rc = resolve(args, p);
+    int rc = resolve(args, p);
     if (rc != PEC_OK) return rc;
     if (p.total_rows == 0) return PEC_OK;   // nothing to write
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (!p.cu_seqlens) {
+        // Rows below the subset's first key see nothing under the causal mask (and no row sees anything of an
+        // empty subset).  Whole 256-row tiles of such rows get no CTA: an in-place merge leaves them as they
+        // are, any other call has them filled (zero / -inf, or a copy of the incoming state).
+        int64_t first_vis = INT64_MAX;
+        for (int t = 0; t < p.n_iv; ++t) first_vis = p.iv_lo[t] < first_vis ? p.iv_lo[t] : first_vis;
+        if (p.n_iv > 0 && !p.causal) first_vis = 0;
+        const bool in_place = p.acc_o && static_cast<const void *>(p.acc_o) == p.o;
+        int kept = 0;
+        for (int s = 0; s < p.n_qseg; ++s) {
+            int64_t lo = p.q_lo[s];
+            const int64_t hi = p.q_hi[s];
+            const int64_t blind_end = first_vis < lo ? lo : (first_vis > hi ? hi : first_vis);
+            int64_t cut = lo + ((blind_end - lo) / kBlockMBf16) * kBlockMBf16;
+            if (blind_end == hi) cut = hi;                 // the whole segment sees nothing
+            if (cut > lo && !in_place) {
+                rc = launch_fill_rows(p, lo - p.out_pos0, cut - p.out_pos0, stream);
+                if (rc != PEC_OK) return rc;
+            }
+            lo = cut;
+            if (hi > lo) { p.q_lo[kept] = lo; p.q_hi[kept] = hi; ++kept; }
+        }
+        p.n_qseg = kept;
+        if (kept == 0) return PEC_OK;
+    }
     if (args->in_dtype != PEC_BF16) return launch_attn_f32(p, stream);
     return launch_attn_prefill_bf16(p, stream);
 }

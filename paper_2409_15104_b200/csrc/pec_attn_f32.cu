@@ -6,6 +6,7 @@
 // rows ty*4..+3 and columns tx+16*j of each 64-key tile, and output rows ty*4..+3 with channels
 // tx*4..+3 and 64+tx*4..+3.  Q, K, V tiles and the probability tile are staged in shared memory.
 #include <cuda_runtime.h>
+#include "pec_host.h"
 #include "pec_internal.h"
 #include "pec_tile.cuh"
 
@@ -147,31 +148,67 @@ attn_f32_kernel(const AttnParams p)
         }
     }
 
-    // epilogue: O / l, LSE = ln 2 * m + ln l (m holds log2-scaled scores)
+    // epilogue: O / l, LSE = ln 2 * m + ln l (m holds log2-scaled scores); with an incoming state the
+    // row's own result is merged into it by the LSE rule first (online softmax across launches).
     float *o = static_cast<float *>(p.o);
     const int64_t out_row0 = job.out_row0;
+    const bool in_place = p.acc_o != nullptr && static_cast<const void *>(p.acc_o) == p.o;
+    // The 16 threads of a row all need the row's incoming LSE, and lse may be that very buffer: every
+    // read comes before the barrier, every write after it.
+    float la_in[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = ty * 4 + i;
+        la_in[i] = (p.acc_o != nullptr && r < job.n_rows) ? p.acc_lse[(out_row0 + r) * p.Hq + h] : -INFINITY;
+    }
+    __syncthreads();
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int r = ty * 4 + i;
         if (r >= job.n_rows) continue;
         const bool empty = (l_run[i] == 0.f);
-        const float inv = empty ? 0.f : 1.f / l_run[i];
-        float *dst = o + ((out_row0 + r) * p.Hq + h) * kHeadDim;
-        *reinterpret_cast<float4 *>(dst + tx * 4) = make_float4(acc[i][0] * inv, acc[i][1] * inv, acc[i][2] * inv, acc[i][3] * inv);
-        *reinterpret_cast<float4 *>(dst + 64 + tx * 4) = make_float4(acc[i][4] * inv, acc[i][5] * inv, acc[i][6] * inv, acc[i][7] * inv);
-        if (tx == 0)
-            p.lse[(out_row0 + r) * p.Hq + h] = empty ? -INFINITY : m_run[i] * 0.6931471805599453f + logf(l_run[i]);
+        if (empty && in_place) continue;                       // the row gained no key: its state stays
+        float c_own = empty ? 0.f : 1.f / l_run[i], c_acc = 0.f;
+        float lse_row = empty ? -INFINITY : m_run[i] * 0.6931471805599453f + logf(l_run[i]);
+        const int64_t item = (out_row0 + r) * p.Hq + h;
+        float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+        if (p.acc_o != nullptr) {
+            const float la = la_in[i];
+            const float mx = fmaxf(lse_row, la);
+            if (mx != -INFINITY) {
+                const float e_own = empty ? 0.f : expf(lse_row - mx), e_acc = (la == -INFINITY) ? 0.f : expf(la - mx);
+                const float inv_tot = 1.f / (e_own + e_acc);
+                c_own *= e_own * inv_tot;
+                c_acc = e_acc * inv_tot;
+                lse_row = mx + logf(e_own + e_acc);
+            }
+            if (c_acc != 0.f) {
+                a0 = *reinterpret_cast<const float4 *>(p.acc_o + item * kHeadDim + tx * 4);
+                a1 = *reinterpret_cast<const float4 *>(p.acc_o + item * kHeadDim + 64 + tx * 4);
+            }
+        }
+        float *dst = o + item * kHeadDim;
+        *reinterpret_cast<float4 *>(dst + tx * 4) = make_float4(fmaf(c_acc, a0.x, acc[i][0] * c_own), fmaf(c_acc, a0.y, acc[i][1] * c_own),
+                                                                fmaf(c_acc, a0.z, acc[i][2] * c_own), fmaf(c_acc, a0.w, acc[i][3] * c_own));
+        *reinterpret_cast<float4 *>(dst + 64 + tx * 4) = make_float4(fmaf(c_acc, a1.x, acc[i][4] * c_own), fmaf(c_acc, a1.y, acc[i][5] * c_own),
+                                                                     fmaf(c_acc, a1.z, acc[i][6] * c_own), fmaf(c_acc, a1.w, acc[i][7] * c_own));
+        if (tx == 0) p.lse[item] = lse_row;
     }
 }
 
 int launch_attn_f32(const AttnParams &p, cudaStream_t stream)
 {
-    if (cudaFuncSetAttribute(attn_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF32Smem) != cudaSuccess) {
+    static unsigned char ready[host::kMaxDevices] = {};
+    static std::mutex ready_mutex;
+    if (!host::once_per_device(ready, ready_mutex, [] {
+            return cudaFuncSetAttribute(attn_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kF32Smem) == cudaSuccess; })) {
         set_error("pec_prefill_attn: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
         return PEC_ERR_CUDA;
     }
-    int64_t tiles = (p.total_rows + kBM - 1) / kBM;
-    if (p.cu_seqlens) tiles += p.B;        // each request may end in a ragged tile
+    int64_t tiles = 0;
+    if (p.cu_seqlens) tiles = p.worklist ? p.n_items : (p.total_rows + kBM - 1) / kBM + p.B;   // each request may end in a ragged tile
+    else for (int s = 0; s < p.n_qseg; ++s) tiles += (p.q_hi[s] - p.q_lo[s] + kBM - 1) / kBM;
+    if (tiles == 0) return PEC_OK;
     if (tiles > 0x7fffffff || p.Hq > 65535) { set_error("pec_prefill_attn: grid too large"); return PEC_ERR_UNSUPPORTED; }
     dim3 grid((unsigned)tiles, (unsigned)p.Hq);
     attn_f32_kernel<<<grid, kF32Threads, kF32Smem, stream>>>(p);

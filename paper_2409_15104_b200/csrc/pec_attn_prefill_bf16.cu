@@ -27,6 +27,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include "pec_host.h"
 #include "pec_internal.h"
 #include "pec_sm100.cuh"
 #include "pec_tile.cuh"
@@ -48,8 +49,6 @@ constexpr uint32_t kKeyHalfBytes = kHalf * 128;            // 64 rows of a box (
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColP = 128, kColO = 256;    // P: + 64 * stage; O: + 128 * stage
 constexpr float kRescaleThreshold = 8.0f;                  // log2 units
-constexpr long long kWaitCycles = 2000000000LL;            // bounded waits give up after ~1 s
-constexpr uint32_t kSuspendNs = 2000;                      // a waiting thread sleeps in the barrier unit this long per try
 
 // What a CTA works on, worked out once by thread 0 and shared through shared memory.  All rows and
 // positions fit in 32 bits (the host rejects larger problems).
@@ -76,20 +75,11 @@ struct Shared {
 };
 constexpr size_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*alignment slack*/ + sizeof(Shared);
 
-// Bounded mbarrier wait.  Returns false (and raises the abort flag / status word) on expiry.
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *sh, int32_t *status)
+// Bounded mbarrier wait (the limit is a launch parameter).  Returns false (and raises the abort flag /
+// status word) on expiry.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *sh, const AttnParams &p)
 {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait_suspend(bar, parity, kSuspendNs)) {
-        if (sh->abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
-            sh->abort_flag = 1;
-            if (status) atomicExch(status, (int)PEC_ERR_TIMEOUT);
-            return false;
-        }
-    }
-    return true;
+    return mbar_wait_bounded(bar, parity, &sh->abort_flag, p.status, p.wait_cycles, (int)PEC_ERR_TIMEOUT);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -115,7 +105,8 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     // stays in registers.)
     TileJob job;
     bool job_found = false;
-    if (warp == kLoadWarp) job_found = locate_tile_warp(p, (int64_t)gridDim.x - 1 - blockIdx.x, kBlockM, job);   // whole warp
+    if (warp == kLoadWarp)                                    // whole warp; a work-list is sorted already
+        job_found = locate_tile_warp(p, p.worklist ? (int64_t)blockIdx.x : (int64_t)gridDim.x - 1 - blockIdx.x, kBlockM, job);
     if (tid == kLoadWarp * 32) {
         Geom g = {};
         g.found = job_found ? 1 : 0;
@@ -200,7 +191,8 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             for (int i = 2; i < 2 * n_max; ++i) {              // items: K(0), V(0) (loaded above), K(1), V(1), ...
                 const int slot = i % kStages, fill = i / kStages;
                 if (sh->abort_flag) break;
-                if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p.status)) break;
+                if (p.test_skip_last_load && i == 2 * n_max - 1) break;   // test hook: the issuers' wait for V(last) runs out
+                if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p)) break;
                 const int jt = i >> 1, c0 = sh->g.cnt[0];
                 const int krow = sh->g.kv_row0 + (jt < c0 ? sh->g.lo[0] + jt * kTile : sh->g.lo[1] + (jt - c0) * kTile);
                 const void *map = (i & 1) ? (const void *)&tm_v : (const void *)&tm_k;
@@ -226,7 +218,7 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kTile, 0, 0);
             constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, kHeadDim, 0, 1);
             auto wait_u = [&](uint64_t *bar, uint32_t parity) {
-                return __all_sync(0xffffffffu, wait_bar(smem_u32(bar), parity, sh, p.status));
+                return __all_sync(0xffffffffu, wait_bar(smem_u32(bar), parity, sh, p));
             };
             auto kv_wait = [&](int item) { return wait_u(&sh->kv_full[item % kStages], (item / kStages) & 1); };
             auto kv_release = [&](int item) { if (leader) tc_commit(smem_u32(&sh->kv_empty[item % kStages])); };
@@ -330,13 +322,15 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             iv_mine[t] = (p.causal && my_pos + 1 < hi_t) ? my_pos + 1 : hi_t;
         }
         int k0 = sh->g.lo[0], cur = 0;
+        const int rows_valid = sh->g.rows[st] - quarter * 32;                   // of this warp's 32 rows
+        const int64_t row0 = (int64_t)sh->g.out_row0 + st * kTile + quarter * 32;
 
         float m_ref = -INFINITY, l_run = 0.f;                // m_ref in log2 units of the scaled scores
         bool ok = true;
         for (int j = 0; j < n_t && ok; ++j, k0 += kTile) {
             if (j == t0) { cur = 1; k0 = sh->g.lo[1]; }
             uint32_t r[kTile];
-            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->s_full[st]), j & 1, sh, p.status));   // warp-uniform
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->s_full[st]), j & 1, sh, p));   // warp-uniform
             if (!ok) break;
             tc_fence_after();
             tmem_ld128(tS, r);
@@ -344,6 +338,12 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->s_taken[st]));
+            // Last tile: start pulling this row of the incoming state towards the L2 (4 x 128 bytes).
+            if (p.acc_o != nullptr && j == n_t - 1 && lane < rows_valid) {
+                const float *src = p.acc_o + ((row0 + lane) * p.Hq + h) * kHeadDim;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) prefetch_l2(src + 32 * c);
+            }
             // Mask only when some row of this stage cannot see the whole tile.
             const bool masked = k0 + kTile > (cur ? iv_full[1] : iv_full[0]);
             if (masked) {
@@ -374,7 +374,7 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             if (j > 0 && __any_sync(0xffffffffu, grow)) {
                 // O still receives P(j-1) V: wait for that product (phase j-1 of the stage's PV barrier; PV(j)
                 // cannot be issued before this warp hands P(j) over, so the phase is unambiguous).
-                ok = __all_sync(0xffffffffu, wait_bar(bar_pv, (j - 1) & 1, sh, p.status));
+                ok = __all_sync(0xffffffffu, wait_bar(bar_pv, (j - 1) & 1, sh, p));
                 if (!ok) break;
                 pv_waited = true;
                 tc_fence_after();
@@ -406,7 +406,7 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             l_run += s01.x + s01.y;
             // P(j-1) is read by its product until that is done.
             if (!pv_waited) {
-                ok = __all_sync(0xffffffffu, wait_bar(bar_pv, (j - 1) & 1, sh, p.status));
+                ok = __all_sync(0xffffffffu, wait_bar(bar_pv, (j - 1) & 1, sh, p));
                 if (!ok) break;
                 tc_fence_after();
             }
@@ -418,60 +418,63 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             if (lane == 0) mbar_arrive(smem_u32(&sh->p_ready[st]));
         }
 
-        // Epilogue: O / l and LSE = ln2 * m + ln l; rows without any visible key give 0 and -inf.
+        // Epilogue: O / l and LSE = ln2 * m + ln l; rows without any visible key give 0 and -inf.  With an
+        // incoming state (acc_o, acc_lse) the stage's own result is merged into it by the LSE rule first
+        // (online softmax across launches): out = c_own * O_raw + c_acc * acc.
         // A thread holds one whole row, so storing from registers would touch 32 rows per instruction.
         // Each warp instead stages 32 rows x 256 bytes in its quarter of the stage's Q tile (no longer
         // read once the stage's last product is done; 16-byte chunks XOR-swizzled by row against bank
         // conflicts) and writes it out two rows per instruction, 256 contiguous bytes each.
-        if (ok && n_hf > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->o_final[st]), 0, sh, p.status));
+        if (ok && n_hf > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->o_final[st]), 0, sh, p));
         // A stage without keys never waited for its Q tile: the load must have landed before the tile is reused.
-        if (ok && n_hf == 0 && n_max > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->bar_q[st]), 0, sh, p.status));
+        if (ok && n_hf == 0 && n_max > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->bar_q[st]), 0, sh, p));
         if (ok && sh->g.rows[st] > 0) {
             tc_fence_after();
+            const bool has_acc = p.acc_o != nullptr;
             const bool empty = (l_run == 0.f);
-            const float inv = empty ? 0.f : 1.f / l_run;
-            const int rows_valid = sh->g.rows[st] - quarter * 32;                 // of this warp's 32 rows
-            const int64_t row0 = (int64_t)sh->g.out_row0 + st * kTile + quarter * 32;
+            float c_own = empty ? 0.f : 1.f / l_run, c_acc = 0.f;
+            float lse_row = empty ? -INFINITY : m_ref * 0.6931471805599453f + logf(l_run);
+            if (has_acc) {
+                const float la = lane < rows_valid ? p.acc_lse[(row0 + lane) * p.Hq + h] : -INFINITY;
+                const float mx = fmaxf(lse_row, la);
+                if (mx != -INFINITY) {
+                    const float e_own = empty ? 0.f : expf(lse_row - mx), e_acc = (la == -INFINITY) ? 0.f : expf(la - mx);
+                    const float inv_tot = 1.f / (e_own + e_acc);           // the larger of the two terms is exactly 1
+                    c_own *= e_own * inv_tot;
+                    c_acc = e_acc * inv_tot;
+                    lse_row = mx + logf(e_own + e_acc);
+                }
+            }
+            // An in-place merge has nothing to write where no row of the warp gained a key.
+            const bool in_place = has_acc && static_cast<const void *>(p.acc_o) == p.o;
+            const bool skip = in_place && __all_sync(0xffffffffu, empty || lane >= rows_valid);
             uint8_t *stage_buf = smem_raw + (tiles - raw) + st * kTileBytes + quarter * 8192;
             uint8_t *my_row = stage_buf + lane * 256;
             const int sub = lane >> 4, chunk = lane & 15;                        // read-back: row parity and 16-byte chunk
-            const int n_pass = p.o_is_bf16 ? 1 : 2;                              // 256 bytes of a row per pass
-            const int64_t row_bytes = (int64_t)p.Hq * kHeadDim * (p.o_is_bf16 ? 2 : 4);
-            uint8_t *out = static_cast<uint8_t *>(p.o) + (row0 + sub) * row_bytes + (int64_t)h * kHeadDim * (p.o_is_bf16 ? 2 : 4) + chunk * 16;
-            for (int pass = 0; pass < n_pass; ++pass) {
-                if (p.o_is_bf16) {
+            const int o_esz = p.o_is_bf16 ? 2 : 4;
+            const int64_t row_bytes = (int64_t)p.Hq * kHeadDim * o_esz;
+            uint8_t *out = static_cast<uint8_t *>(p.o) + (row0 + sub) * row_bytes + (int64_t)h * kHeadDim * o_esz;
+            if (skip) {
+                // nothing
+            } else if (!has_acc && p.o_is_bf16) {
+                // One pass: a row is 256 bytes of bf16.
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {                        // 64 channels = 8 chunks of 16 bytes
-                        uint32_t r[64];
-                        if (n_hf == 0) {
-#pragma unroll
-                            for (int i = 0; i < 64; ++i) r[i] = 0u;
-                        } else {
-                            tmem_ld64(tO + half * 64, r);
-                        }
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            uint4 pk;
-                            pk.x = pack_bf16(__uint_as_float(r[8 * i + 0]) * inv, __uint_as_float(r[8 * i + 1]) * inv);
-                            pk.y = pack_bf16(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
-                            pk.z = pack_bf16(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv);
-                            pk.w = pack_bf16(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv);
-                            *reinterpret_cast<uint4 *>(my_row + (((half * 8 + i) ^ (lane & 15)) << 4)) = pk;
-                        }
-                    }
-                } else {
-                    uint32_t r[64];                                               // 64 channels = 16 chunks of 16 bytes
+                for (int half = 0; half < 2; ++half) {                        // 64 channels = 8 chunks of 16 bytes
+                    uint32_t r[64];
                     if (n_hf == 0) {
 #pragma unroll
                         for (int i = 0; i < 64; ++i) r[i] = 0u;
                     } else {
-                        tmem_ld64(tO + pass * 64, r);
+                        tmem_ld64(tO + half * 64, r);
                     }
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float4 f = make_float4(__uint_as_float(r[4 * i]) * inv, __uint_as_float(r[4 * i + 1]) * inv,
-                                                     __uint_as_float(r[4 * i + 2]) * inv, __uint_as_float(r[4 * i + 3]) * inv);
-                        *reinterpret_cast<float4 *>(my_row + ((i ^ (lane & 15)) << 4)) = f;
+                    for (int i = 0; i < 8; ++i) {
+                        uint4 pk;
+                        pk.x = pack_bf16(__uint_as_float(r[8 * i + 0]) * c_own, __uint_as_float(r[8 * i + 1]) * c_own);
+                        pk.y = pack_bf16(__uint_as_float(r[8 * i + 2]) * c_own, __uint_as_float(r[8 * i + 3]) * c_own);
+                        pk.z = pack_bf16(__uint_as_float(r[8 * i + 4]) * c_own, __uint_as_float(r[8 * i + 5]) * c_own);
+                        pk.w = pack_bf16(__uint_as_float(r[8 * i + 6]) * c_own, __uint_as_float(r[8 * i + 7]) * c_own);
+                        *reinterpret_cast<uint4 *>(my_row + (((half * 8 + i) ^ (lane & 15)) << 4)) = pk;
                     }
                 }
                 __syncwarp();
@@ -482,13 +485,69 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     const int row = 2 * rr + sub;
                     val[rr] = *reinterpret_cast<const uint4 *>(stage_buf + row * 256 + ((chunk ^ (row & 15)) << 4));
                 }
-                uint8_t *dst = out + (p.o_is_bf16 ? 0 : pass * 256);
+                uint8_t *dst = out + chunk * 16;
 #pragma unroll
                 for (int rr = 0; rr < 16; ++rr, dst += 2 * row_bytes)
                     if (2 * rr + sub < rows_valid) *reinterpret_cast<uint4 *>(dst) = val[rr];
-                __syncwarp();
+            } else {
+                // Two passes of 64 channels staged as fp32 (256 bytes of a row each).
+                const float *acc_base = has_acc ? p.acc_o + ((row0 + sub) * p.Hq + h) * kHeadDim + chunk * 4 : nullptr;
+#pragma unroll 1
+                for (int pass = 0; pass < 2; ++pass) {
+                    // The incoming state's loads go first: their latency runs under the TMEM read and the staging.
+                    float4 inc[16];
+                    if (has_acc) {
+                        const float *src = acc_base + pass * 64;
+#pragma unroll
+                        for (int rr = 0; rr < 16; ++rr, src += 2 * (int64_t)p.Hq * kHeadDim) {
+                            inc[rr] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (2 * rr + sub < rows_valid) inc[rr] = *reinterpret_cast<const float4 *>(src);
+                        }
+                    }
+                    uint32_t r[64];                                               // 64 channels = 16 chunks of 16 bytes
+                    if (n_hf == 0) {
+#pragma unroll
+                        for (int i = 0; i < 64; ++i) r[i] = 0u;
+                    } else {
+                        tmem_ld64(tO + pass * 64, r);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float4 f = make_float4(__uint_as_float(r[4 * i]) * c_own, __uint_as_float(r[4 * i + 1]) * c_own,
+                                                     __uint_as_float(r[4 * i + 2]) * c_own, __uint_as_float(r[4 * i + 3]) * c_own);
+                        *reinterpret_cast<float4 *>(my_row + ((i ^ (lane & 15)) << 4)) = f;
+                    }
+                    __syncwarp();
+                    float4 val[16];
+#pragma unroll
+                    for (int rr = 0; rr < 16; ++rr) {
+                        const int row = 2 * rr + sub;
+                        val[rr] = *reinterpret_cast<const float4 *>(stage_buf + row * 256 + ((chunk ^ (row & 15)) << 4));
+                    }
+                    if (has_acc) {
+#pragma unroll
+                        for (int rr = 0; rr < 16; ++rr) {
+                            const float w = __shfl_sync(0xffffffffu, c_acc, 2 * rr + sub);   // the row's weight sits with its owner
+                            val[rr].x = fmaf(w, inc[rr].x, val[rr].x); val[rr].y = fmaf(w, inc[rr].y, val[rr].y);
+                            val[rr].z = fmaf(w, inc[rr].z, val[rr].z); val[rr].w = fmaf(w, inc[rr].w, val[rr].w);
+                        }
+                    }
+                    if (p.o_is_bf16) {
+                        uint8_t *dst = out + pass * 128 + chunk * 8;
+#pragma unroll
+                        for (int rr = 0; rr < 16; ++rr, dst += 2 * row_bytes)
+                            if (2 * rr + sub < rows_valid)
+                                *reinterpret_cast<uint2 *>(dst) = make_uint2(pack_bf16(val[rr].x, val[rr].y), pack_bf16(val[rr].z, val[rr].w));
+                    } else {
+                        uint8_t *dst = out + pass * 256 + chunk * 16;
+#pragma unroll
+                        for (int rr = 0; rr < 16; ++rr, dst += 2 * row_bytes)
+                            if (2 * rr + sub < rows_valid) *reinterpret_cast<float4 *>(dst) = val[rr];
+                    }
+                    __syncwarp();
+                }
             }
-            if (lane < rows_valid) p.lse[(row0 + lane) * p.Hq + h] = empty ? -INFINITY : m_ref * 0.6931471805599453f + logf(l_run);
+            if (!skip && lane < rows_valid) p.lse[(row0 + lane) * p.Hq + h] = lse_row;
         }
     }
 
@@ -498,37 +557,6 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 }
 
 // ------------------------------------------------------------------------------------------ host
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
-// [rows, heads, 128] bf16 tensor with element strides (stride_t, stride_h); box = 64 channels x 1 head x 128 rows.
-static bool make_map(CUtensorMap *map, const void *base, int64_t rows, int32_t heads, int64_t stride_t, int64_t stride_h)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)heads, (cuuint64_t)(rows > 0 ? rows : 1)};
-    cuuint64_t strides[2] = {(cuuint64_t)stride_h * 2, (cuuint64_t)stride_t * 2};
-    cuuint32_t box[3] = {64, 1, 128};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace pf
 
 int launch_attn_prefill_bf16(const AttnParams &p, cudaStream_t stream)
@@ -536,39 +564,45 @@ int launch_attn_prefill_bf16(const AttnParams &p, cudaStream_t stream)
     using namespace pf;
     if (!p.status) { set_error("pec_prefill_attn: the bf16 path needs a status word"); return PEC_ERR_INVALID_ARG; }
     if (p.splits != 1) { set_error("pec_prefill_attn: this kernel takes no split launches"); return PEC_ERR_INVALID_ARG; }
-    // Rows the maps may touch: queries up to the chunk end, keys up to the end of the visible subset.
-    int64_t q_rows, kv_rows;
-    if (p.cu_seqlens) { q_rows = p.total_rows; kv_rows = p.total_rows; }
-    else {
-        q_rows = p.chunk_start + p.chunk_len;
-        kv_rows = 0;
+    // Rows the maps may touch: queries up to the last segment's end, keys up to the end of the visible subset.
+    int64_t q_rows = 0, kv_rows = 0, tiles = 0;
+    if (p.cu_seqlens) {
+        q_rows = p.total_rows; kv_rows = p.total_rows;
+        tiles = p.worklist ? p.n_items : (p.total_rows + kBlockM - 1) / kBlockM + p.B;   // without a list every request may end in a ragged tile
+    } else {
+        for (int s = 0; s < p.n_qseg; ++s) {
+            q_rows = p.q_hi[s] > q_rows ? p.q_hi[s] : q_rows;
+            tiles += (p.q_hi[s] - p.q_lo[s] + kBlockM - 1) / kBlockM;
+        }
         for (int t = 0; t < p.n_iv; ++t) kv_rows = p.iv_hi[t] > kv_rows ? p.iv_hi[t] : kv_rows;
     }
+    if (tiles == 0) return PEC_OK;
     if (q_rows >= ((int64_t)1 << 31) || kv_rows >= ((int64_t)1 << 31)) {
         set_error("pec_prefill_attn: more than 2^31 rows unsupported");
         return PEC_ERR_UNSUPPORTED;
     }
     CUtensorMap tm_q, tm_k, tm_v;
-    if (!make_map(&tm_q, p.q, q_rows, p.Hq, p.q_stride_t, p.q_stride_h) ||
-        !make_map(&tm_k, p.k, kv_rows, p.Hkv, p.k_stride_t, p.k_stride_h) ||
-        !make_map(&tm_v, p.v, kv_rows, p.Hkv, p.v_stride_t, p.v_stride_h)) {
+    if (!host::make_qkv_map(&tm_q, p.q, q_rows, p.Hq, p.q_stride_t, p.q_stride_h) ||
+        !host::make_qkv_map(&tm_k, p.k, kv_rows, p.Hkv, p.k_stride_t, p.k_stride_h) ||
+        !host::make_qkv_map(&tm_v, p.v, kv_rows, p.Hkv, p.v_stride_t, p.v_stride_h)) {
         set_error("pec_prefill_attn: cuTensorMapEncodeTiled failed (driver too old, or strides/addresses not encodable)");
         return PEC_ERR_CUDA;
     }
-    if (cudaFuncSetAttribute(attn_prefill_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) {
-        set_error("pec_prefill_attn: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
+    // Once per device: raise the shared-memory limit, and check that the launch allocation (registers per
+    // thread x threads) covers the split in which the softmax warpgroups take registers the third gives up.
+    static unsigned char ready[host::kMaxDevices] = {};
+    static std::mutex ready_mutex;
+    const bool ok = host::once_per_device(ready, ready_mutex, [] {
+        if (cudaFuncSetAttribute(attn_prefill_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) return false;
+        cudaFuncAttributes attr;
+        return cudaFuncGetAttributes(&attr, attn_prefill_bf16_kernel) == cudaSuccess &&
+               attr.numRegs * kThreads >= kSoftmaxWarps * 32 * kSoftmaxRegs + (kThreads - kSoftmaxWarps * 32) * kLightRegs;
+    });
+    if (!ok) {
+        (void)cudaGetLastError();
+        set_error("pec_prefill_attn: kernel set-up failed (shared-memory limit, or the register allocation does not cover the warp-role split)");
         return PEC_ERR_CUDA;
     }
-    // The softmax warpgroups take registers the third warpgroup gives up; that only works when the
-    // launch allocation (registers per thread x threads) covers the new split.
-    cudaFuncAttributes attr;
-    if (cudaFuncGetAttributes(&attr, attn_prefill_bf16_kernel) != cudaSuccess ||
-        attr.numRegs * kThreads < kSoftmaxWarps * 32 * kSoftmaxRegs + (kThreads - kSoftmaxWarps * 32) * kLightRegs) {
-        set_error("pec_prefill_attn: kernel register allocation too small for the warp-role register split");
-        return PEC_ERR_CUDA;
-    }
-    int64_t tiles = (p.total_rows + kBlockM - 1) / kBlockM;
-    if (p.cu_seqlens) tiles += p.B;
     if (tiles > 0x7fffffff || p.Hq > 65535) { set_error("pec_prefill_attn: grid too large"); return PEC_ERR_UNSUPPORTED; }
     dim3 grid((unsigned)tiles, (unsigned)p.Hq, 1);
     attn_prefill_bf16_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, p);

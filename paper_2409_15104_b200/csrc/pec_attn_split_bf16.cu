@@ -21,6 +21,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include "pec_host.h"
 #include "pec_internal.h"
 #include "pec_sm100.cuh"
 #include "pec_tile.cuh"
@@ -40,8 +41,6 @@ constexpr uint32_t kTileBytes = 2 * kHalfTileBytes;        // 128 x 128 bf16
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;                 // + 128 * stage
 constexpr float kRescaleThreshold = 8.0f;                  // log2 units
-constexpr long long kWaitCycles = 2000000000LL;            // bounded waits give up after ~1 s
-constexpr uint32_t kSuspendNs = 2000;                      // a waiting thread sleeps in the barrier unit this long per try
 
 // What a CTA works on, worked out once by thread 0 and shared through shared memory.  All rows and
 // positions fit in 32 bits (the host rejects larger problems).
@@ -67,20 +66,11 @@ struct Shared {
 };
 constexpr size_t kSmemBytes = (2 + kStages) * kTileBytes + 1024 /*alignment slack*/ + sizeof(Shared);
 
-// Bounded mbarrier wait.  Returns false (and raises the abort flag / status word) on expiry.
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *sh, int32_t *status)
+// Bounded mbarrier wait (the limit is a launch parameter).  Returns false (and raises the abort flag /
+// status word) on expiry.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *sh, const AttnParams &p)
 {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait_suspend(bar, parity, kSuspendNs)) {
-        if (sh->abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
-            sh->abort_flag = 1;
-            if (status) atomicExch(status, (int)PEC_ERR_TIMEOUT);
-            return false;
-        }
-    }
-    return true;
+    return mbar_wait_bounded(bar, parity, &sh->abort_flag, p.status, p.wait_cycles, (int)PEC_ERR_TIMEOUT);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -168,7 +158,7 @@ attn_split_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             int filled = 0;                                    // ring items issued so far
             auto load_tile = [&](const void *map, int krow) {
                 const int slot = filled % kStages, fill = filled / kStages;
-                if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p.status)) return false;
+                if (fill > 0 && !wait_bar(smem_u32(&sh->kv_empty[slot]), (fill - 1) & 1, sh, p)) return false;
                 const uint32_t dst = sRing + slot * kTileBytes, bar = smem_u32(&sh->kv_full[slot]);
                 mbar_arrive_expect_tx(bar, kTileBytes);
                 tma_load_3d(dst, map, bar, 0, kvh, krow);
@@ -200,7 +190,7 @@ attn_split_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kTile, 0, 0);
             constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, kHeadDim, 0, 1);
             auto kv_wait = [&](int item) {
-                return wait_bar(smem_u32(&sh->kv_full[item % kStages]), (item / kStages) & 1, sh, p.status);
+                return wait_bar(smem_u32(&sh->kv_full[item % kStages]), (item / kStages) & 1, sh, p);
             };
             auto kv_release = [&](int item) { tc_commit(smem_u32(&sh->kv_empty[item % kStages])); };
             // S_st = Q_st K^T: both operands K-major; 8 steps of 16 channels, 4 per 64-channel half tile
@@ -225,7 +215,7 @@ attn_split_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             };
 
             const int n_st[2] = {sh->g.n[0], sh->g.n[1]};
-            bool ok = wait_bar(smem_u32(&sh->bar_q), 0, sh, p.status);
+            bool ok = wait_bar(smem_u32(&sh->bar_q), 0, sh, p);
             if (ok) {
                 // Every ring item has one consumer; items arrive in the order used here.
                 int item = 0;
@@ -240,7 +230,7 @@ attn_split_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 #pragma unroll
                     for (int st = 0; st < 2 && ok; ++st) {
                         if (j < n_st[st]) {
-                            ok = wait_bar(smem_u32(&sh->p_ready[st]), j & 1, sh, p.status) && kv_wait(item);   // P_st(j), V_st(j)
+                            ok = wait_bar(smem_u32(&sh->p_ready[st]), j & 1, sh, p) && kv_wait(item);   // P_st(j), V_st(j)
                             if (!ok) break;
                             tc_fence_after();
                             issue_pv(st, item, j > 0);
@@ -283,7 +273,7 @@ attn_split_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         float m_ref = -INFINITY, l_run = 0.f;                // m_ref in log2 units of the scaled scores
         bool ok = true;
         for (int j = 0; j < n_mine; ++j, k0 += kTile) {
-            ok = __all_sync(0xffffffffu, wait_bar(bar_s, j & 1, sh, p.status));     // warp-uniform
+            ok = __all_sync(0xffffffffu, wait_bar(bar_s, j & 1, sh, p));     // warp-uniform
             if (!ok) break;
             tc_fence_after();
 
@@ -351,7 +341,7 @@ attn_split_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         }
 
         // Epilogue: O / l and LSE = ln2 * m + ln l; rows without any visible key give 0 and -inf.
-        if (ok && n_mine > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->o_final[st]), 0, sh, p.status));
+        if (ok && n_mine > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->o_final[st]), 0, sh, p));
         if (ok && sh->g.rows[st] > 0) {
             tc_fence_after();
             const bool valid = row_in_tile < sh->g.rows[st];
@@ -398,37 +388,6 @@ attn_split_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 }
 
 // ------------------------------------------------------------------------------------------ host
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
-// [rows, heads, 128] bf16 tensor with element strides (stride_t, stride_h); box = 64 channels x 1 head x 128 rows.
-static bool make_map(CUtensorMap *map, const void *base, int64_t rows, int32_t heads, int64_t stride_t, int64_t stride_h)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)heads, (cuuint64_t)(rows > 0 ? rows : 1)};
-    cuuint64_t strides[2] = {(cuuint64_t)stride_h * 2, (cuuint64_t)stride_t * 2};
-    cuuint32_t box[3] = {64, 1, 128};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace splitk
 
 int launch_attn_split_bf16(const AttnParams &p, cudaStream_t stream)
@@ -437,7 +396,7 @@ int launch_attn_split_bf16(const AttnParams &p, cudaStream_t stream)
     if (!p.status) { set_error("pec_decode_attn: the bf16 path needs a status word"); return PEC_ERR_INVALID_ARG; }
     // Rows the maps may touch: queries up to the chunk end, keys up to the end of the visible subset.
     if (p.cu_seqlens) { set_error("pec_decode_attn: packed batches are not split"); return PEC_ERR_INVALID_ARG; }
-    const int64_t q_rows = p.chunk_start + p.chunk_len;
+    const int64_t q_rows = p.q_hi[0];
     int64_t kv_rows = 0;
     for (int t = 0; t < p.n_iv; ++t) kv_rows = p.iv_hi[t] > kv_rows ? p.iv_hi[t] : kv_rows;
     if (q_rows >= ((int64_t)1 << 31) || kv_rows >= ((int64_t)1 << 31)) {
@@ -445,22 +404,25 @@ int launch_attn_split_bf16(const AttnParams &p, cudaStream_t stream)
         return PEC_ERR_UNSUPPORTED;
     }
     CUtensorMap tm_q, tm_k, tm_v;
-    if (!make_map(&tm_q, p.q, q_rows, p.Hq, p.q_stride_t, p.q_stride_h) ||
-        !make_map(&tm_k, p.k, kv_rows, p.Hkv, p.k_stride_t, p.k_stride_h) ||
-        !make_map(&tm_v, p.v, kv_rows, p.Hkv, p.v_stride_t, p.v_stride_h)) {
+    if (!host::make_qkv_map(&tm_q, p.q, q_rows, p.Hq, p.q_stride_t, p.q_stride_h) ||
+        !host::make_qkv_map(&tm_k, p.k, kv_rows, p.Hkv, p.k_stride_t, p.k_stride_h) ||
+        !host::make_qkv_map(&tm_v, p.v, kv_rows, p.Hkv, p.v_stride_t, p.v_stride_h)) {
         set_error("pec_decode_attn: cuTensorMapEncodeTiled failed (driver too old, or strides/addresses not encodable)");
         return PEC_ERR_CUDA;
     }
-    if (cudaFuncSetAttribute(attn_split_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) {
-        set_error("pec_decode_attn: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
-        return PEC_ERR_CUDA;
-    }
-    // The softmax warpgroups take registers the third warpgroup gives up; that only works when the
-    // launch allocation (registers per thread x threads) covers the new split.
-    cudaFuncAttributes attr;
-    if (cudaFuncGetAttributes(&attr, attn_split_bf16_kernel) != cudaSuccess ||
-        attr.numRegs * kThreads < kSoftmaxWarps * 32 * kSoftmaxRegs + (kThreads - kSoftmaxWarps * 32) * kLightRegs) {
-        set_error("pec_decode_attn: kernel register allocation too small for the warp-role register split");
+    // Once per device: raise the shared-memory limit, and check that the launch allocation (registers per
+    // thread x threads) covers the split in which the softmax warpgroups take registers the third gives up.
+    static unsigned char ready[host::kMaxDevices] = {};
+    static std::mutex ready_mutex;
+    const bool ok = host::once_per_device(ready, ready_mutex, [] {
+        if (cudaFuncSetAttribute(attn_split_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess) return false;
+        cudaFuncAttributes attr;
+        return cudaFuncGetAttributes(&attr, attn_split_bf16_kernel) == cudaSuccess &&
+               attr.numRegs * kThreads >= kSoftmaxWarps * 32 * kSoftmaxRegs + (kThreads - kSoftmaxWarps * 32) * kLightRegs;
+    });
+    if (!ok) {
+        (void)cudaGetLastError();
+        set_error("pec_decode_attn: kernel set-up failed (shared-memory limit, or the register allocation does not cover the warp-role split)");
         return PEC_ERR_CUDA;
     }
     const int64_t tiles = (p.total_rows + kBlockM - 1) / kBlockM;

@@ -114,7 +114,8 @@ static int run_decode(const pec_decode_args *a, const DecodeShape &shape, void *
     p.v_stride_t = a->v_stride_t; p.v_stride_h = a->v_stride_h;
     p.Hq = a->Hkv; p.Hkv = a->Hkv; p.group = 1;
     p.cu_seqlens = nullptr; p.B = 1;
-    p.chunk_start = 0; p.chunk_len = g; p.total_rows = g;
+    p.q_lo[0] = 0; p.q_hi[0] = g; p.n_qseg = 1; p.out_pos0 = 0; p.total_rows = g;
+    p.wait_cycles = wait_limit_cycles();
     p.iv_lo[0] = a->kv_lo; p.iv_hi[0] = a->kv_hi; p.iv_lo[1] = p.iv_hi[1] = 0;
     p.n_iv = a->kv_hi > a->kv_lo ? 1 : 0;
     p.causal = 0;

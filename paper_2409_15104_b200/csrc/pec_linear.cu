@@ -15,6 +15,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include "pec_host.h"
 #include "pec_internal.h"
 #include "pec_sm100.cuh"
 
@@ -29,7 +30,6 @@ constexpr uint32_t kABytes = kBM * kBK * 2;                 // this CTA's 128 ro
 constexpr uint32_t kWBytes = 128 * kBK * 2;                 // this CTA's half of the 256 rows of w
 constexpr uint32_t kSlotBytes = kABytes + kWBytes;          // 32 KB
 constexpr uint32_t kTmemCols = 256;
-constexpr long long kWaitCycles = 2000000000LL;
 
 struct Shared {
     uint64_t full[kSlots], empty[kSlots], acc_full;
@@ -38,24 +38,17 @@ struct Shared {
 };
 constexpr size_t kSmemBytes = kSlots * kSlotBytes + 1024 + sizeof(Shared);
 
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, Shared *sh, int32_t *status)
+// What the waits of a CTA need: its abort flag, the caller's status word and the wait limit.
+struct WaitCtx { volatile int *abort_flag; int32_t *status; long long limit; };
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const WaitCtx &w)
 {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait_suspend(bar, parity, 2000)) {
-        if (sh->abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
-            sh->abort_flag = 1;
-            if (status) atomicExch(status, (int)PEC_ERR_TIMEOUT);
-            return false;
-        }
-    }
-    return true;
+    return mbar_wait_bounded(bar, parity, w.abort_flag, w.status, w.limit, (int)PEC_ERR_TIMEOUT);
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 2)
 linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-                   __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t band, int32_t *status)
+                   __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t band, int32_t *status,
+              long long wait_cycles, int32_t test_skip_last_load)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -75,6 +68,7 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
     const int64_t m0 = (int64_t)(band_i * band + within % band_pairs) * (2 * kBM) + rank * kBM;
     const int n0 = (within / band_pairs) * kBN;
     const int n_kb = (K + kBK - 1) / kBK;
+    const WaitCtx wctx = {&sh->abort_flag, status, wait_cycles};
 
     if (tid == 0) {
         sh->abort_flag = (status && *reinterpret_cast<volatile int32_t *>(status) != 0) ? 1 : 0;
@@ -100,7 +94,8 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
         if (lane == 0) {
             for (int kb = 0; kb < n_kb; ++kb) {
                 const int slot = kb % kSlots, fill = kb / kSlots;
-                if (fill > 0 && !wait_bar(smem_u32(&sh->empty[slot]), (fill - 1) & 1, sh, status)) break;
+                if (test_skip_last_load && rank == 1 && kb == n_kb - 1) break;   // test hook: the pair's waits for this step run out
+                if (fill > 0 && !wait_bar(smem_u32(&sh->empty[slot]), (fill - 1) & 1, wctx)) break;
                 const uint32_t a = ring + slot * kSlotBytes;
                 const uint32_t bar = leader_addr(smem_u32(&sh->full[slot]));
                 if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[slot]), 2 * kSlotBytes);   // both CTAs' bytes
@@ -115,7 +110,7 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
             bool ok = true;
             for (int kb = 0; kb < n_kb && ok; ++kb) {
                 const int slot = kb % kSlots;
-                ok = wait_bar(smem_u32(&sh->full[slot]), (kb / kSlots) & 1, sh, status);
+                ok = wait_bar(smem_u32(&sh->full[slot]), (kb / kSlots) & 1, wctx);
                 if (!ok) break;
                 const uint32_t a = ring + slot * kSlotBytes, b = a + kABytes;
 #pragma unroll
@@ -128,7 +123,7 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
         }
         __syncwarp();
     } else {
-        const bool ok = __all_sync(0xffffffffu, n_kb == 0 || wait_bar(smem_u32(&sh->acc_full), 0, sh, status));
+        const bool ok = __all_sync(0xffffffffu, n_kb == 0 || wait_bar(smem_u32(&sh->acc_full), 0, wctx));
         if (ok) {
             tc_fence_after();
             const int64_t row = m0 + warp * 32 + lane;
@@ -160,36 +155,6 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
     if (warp == 0) tmem_dealloc_pair(tmem, kTmemCols);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
-// [rows, cols] bf16 matrix, row stride in elements; box = 64 columns x box_rows rows.
-static bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t cols, int64_t stride, int box_rows)
-{
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)stride * 2};
-    cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 }  // namespace lin
 }  // namespace pec
 
@@ -209,11 +174,14 @@ extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_
     }
     if (M == 0) return PEC_OK;
     CUtensorMap tm_x, tm_w;
-    if (!lin::make_map(&tm_x, x, M, K, x_stride, lin::kBM) || !lin::make_map(&tm_w, w, N, K, w_stride, 128)) {
+    if (!host::make_matrix_map(&tm_x, x, M, K, x_stride, lin::kBM) || !host::make_matrix_map(&tm_w, w, N, K, w_stride, 128)) {
         set_error("pec_linear: cuTensorMapEncodeTiled failed");
         return PEC_ERR_CUDA;
     }
-    if (cudaFuncSetAttribute(lin::linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::kSmemBytes) != cudaSuccess) {
+    static unsigned char ready[host::kMaxDevices] = {};
+    static std::mutex ready_mutex;
+    if (!host::once_per_device(ready, ready_mutex, [] {
+            return cudaFuncSetAttribute(lin::linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::kSmemBytes) == cudaSuccess; })) {
         set_error("pec_linear: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
         return PEC_ERR_CUDA;
     }
@@ -225,7 +193,8 @@ extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_
     band = band < 4 ? 4 : (band > 32 ? 32 : band);
     dim3 grid((unsigned)(2 * pairs), (unsigned)gn);           // clusters of two CTAs along x
     lin::linear_kernel<<<grid, lin::kThreads, lin::kSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(
-        tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, (int32_t)band, status);
+        tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, (int32_t)band, status,
+        (long long)wait_limit_cycles(), test_skip_last_load());
     const cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("pec_linear: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;

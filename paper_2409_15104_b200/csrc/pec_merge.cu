@@ -170,6 +170,37 @@ merge_n_kernel(const MergeParts parts, void *o_out, float *lse_out, int64_t item
     }
 }
 
+// Rows of an attention call that no CTA covers because they see no key of the call's subset: the
+// partial of such a row is the merge identity (o = 0, lse = -inf), or - with an incoming state - that
+// state unchanged, rounded to the output type.  One float4 of a row per thread.
+template <bool kOutBf16>
+__global__ void __launch_bounds__(kMergeThreads)
+fill_rows_kernel(void *o, float *lse, const float *__restrict__ acc_o, const float *__restrict__ acc_lse,
+                 int64_t item_lo, int64_t item_hi)
+{
+    const int64_t n4 = (item_hi - item_lo) * (kHeadDim / 4);
+    const int64_t stride = (int64_t)gridDim.x * kMergeThreads;
+    for (int64_t i = (int64_t)blockIdx.x * kMergeThreads + threadIdx.x; i < n4; i += stride) {
+        const int64_t off = item_lo * (kHeadDim / 4) + i;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (acc_o) v = ld_stream(reinterpret_cast<const float4 *>(acc_o) + off);
+        if (kOutBf16) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+            __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t *>(&lo);
+            pk.y = *reinterpret_cast<uint32_t *>(&hi);
+            reinterpret_cast<uint2 *>(o)[off] = pk;
+        } else {
+            reinterpret_cast<float4 *>(o)[off] = v;
+        }
+        if ((i & (kHeadDim / 4 - 1)) == 0) {
+            const int64_t item = item_lo + i / (kHeadDim / 4);
+            lse[item] = acc_lse ? acc_lse[item] : -INFINITY;
+        }
+    }
+}
+
 static int merge_grid(int64_t items, const char *who, int64_t *ctas_out)
 {
     static int sm_count = 0;
@@ -187,6 +218,20 @@ static int merge_grid(int64_t items, const char *who, int64_t *ctas_out)
     int64_t ctas = (n_groups + warps_per_cta - 1) / warps_per_cta;
     const int64_t cap = (int64_t)sm_count * 8;
     *ctas_out = ctas > cap ? cap : ctas;
+    return PEC_OK;
+}
+
+int launch_fill_rows(const AttnParams &p, int64_t row_lo, int64_t row_hi, cudaStream_t stream)
+{
+    if (row_hi <= row_lo) return PEC_OK;
+    const int64_t item_lo = row_lo * p.Hq, item_hi = row_hi * p.Hq;
+    int64_t ctas = 0;
+    const int rc = merge_grid(item_hi - item_lo, "pec_prefill_attn", &ctas);
+    if (rc != PEC_OK) return rc;
+    if (p.o_is_bf16) fill_rows_kernel<true><<<(unsigned)ctas, kMergeThreads, 0, stream>>>(p.o, p.lse, p.acc_o, p.acc_lse, item_lo, item_hi);
+    else             fill_rows_kernel<false><<<(unsigned)ctas, kMergeThreads, 0, stream>>>(p.o, p.lse, p.acc_o, p.acc_lse, item_lo, item_hi);
+    const cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) { set_error("pec_prefill_attn: fill launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;
 }
 

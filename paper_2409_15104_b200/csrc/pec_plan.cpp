@@ -108,6 +108,41 @@ extern "C" int pec_plan_partitions(int64_t seq_len, int32_t num_parts, int64_t c
     return PEC_OK;
 }
 
+extern "C" int pec_plan_worklist(const int32_t *cu_seqlens, int32_t B, int32_t block_m, int32_t block_n, int32_t causal,
+                                 int32_t *items, int64_t items_cap, int64_t *n_items)
+{
+    if (!cu_seqlens || !n_items || B < 0 || block_m < 1 || block_n < 1) {
+        set_error("pec_plan_worklist: need cu_seqlens, n_items, B >= 0 and block sizes >= 1");
+        return PEC_ERR_INVALID_ARG;
+    }
+    int64_t total = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        if (cu_seqlens[b + 1] < cu_seqlens[b]) { set_error("pec_plan_worklist: cu_seqlens decreases at request %d", (int)b); return PEC_ERR_INVALID_ARG; }
+        total += ceil_div((int64_t)cu_seqlens[b + 1] - cu_seqlens[b], block_m);
+    }
+    *n_items = total;
+    if (!items) return PEC_OK;
+    if (items_cap < total) { set_error("pec_plan_worklist: items holds %lld entries, %lld needed", (long long)items_cap, (long long)total); return PEC_ERR_CAPACITY; }
+    struct Entry { int64_t weight; int32_t start, pos0, rows, len; };
+    std::vector<Entry> list;
+    list.reserve((size_t)total);
+    for (int32_t b = 0; b < B; ++b) {
+        const int64_t len = (int64_t)cu_seqlens[b + 1] - cu_seqlens[b];
+        for (int64_t pos0 = 0; pos0 < len; pos0 += block_m) {
+            const int64_t rows = len - pos0 < block_m ? len - pos0 : block_m;
+            const int64_t keys = causal ? pos0 + rows : len;      // the tile's last row sees keys [0, pos0 + rows)
+            list.push_back({ceil_div(keys, block_n), cu_seqlens[b], (int32_t)pos0, (int32_t)rows, (int32_t)len});
+        }
+    }
+    // Entries were generated by request, then by position: a stable sort keeps that order among equal weights.
+    std::stable_sort(list.begin(), list.end(), [](const Entry &x, const Entry &y) { return x.weight > y.weight; });
+    for (size_t i = 0; i < list.size(); ++i) {
+        items[4 * i + 0] = list[i].start; items[4 * i + 1] = list[i].pos0;
+        items[4 * i + 2] = list[i].rows;  items[4 * i + 3] = list[i].len;
+    }
+    return PEC_OK;
+}
+
 // Visible (query, key) pairs between query rows [a, b) and keys [c, d): a key j counts for row i
 // when j <= i (causal) or always.  Rows below the first key see nothing, rows i in [c, d-1) see
 // i + 1 - c keys (an arithmetic series), rows from d - 1 on see all d - c.

@@ -54,6 +54,27 @@ __device__ __forceinline__ bool mbar_try_wait_suspend(uint32_t bar, uint32_t par
     return ok != 0;
 }
 
+// Bounded wait on an mbarrier phase, shared by every kernel of the library.  A waiting thread sleeps
+// in the barrier unit for up to 2 us per try and gives up when `limit_cycles` SM clocks have passed or
+// when another thread of the CTA has raised `*abort_flag` (shared memory).  On expiry it raises the flag
+// itself and stores `timeout_code` in the caller's status word, so that every other wait of the CTA
+// fails at its next try and the CTA reaches its common exit.  Returns false when the wait was given up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
+                                                  long long limit_cycles, int timeout_code)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait_suspend(bar, parity, 2000u)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limit_cycles) {
+            *abort_flag = 1;
+            if (status) atomicExch(status, timeout_code);
+            return false;
+        }
+    }
+    return true;
+}
+
 // ---------------------------------------------------------------- TMA
 // 3-D tiled load: coordinates are (innermost, middle, outermost) in elements.
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, uint32_t bar, int c0, int c1, int c2)
@@ -61,6 +82,10 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, uint
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(tmap), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void prefetch_l2(const void *gptr)
+{
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(gptr) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const void *tmap)
 {
@@ -175,34 +200,6 @@ __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// The same two MMAs with each descriptor passed as its two 32-bit words.  The MMAs of a tile differ
-// only in the start address, so the issuing thread keeps the low word of the tile's descriptor and
-// adds a constant per K step; building a 64-bit descriptor per instruction costs a lone thread more
-// cycles than the MMA occupies the tensor pipe.
-constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);   // SBO = 1024 bytes, version 1, SWIZZLE_128B
-__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes)
-{
-    return ((saddr >> 4) & 0x3fffu) | ((lbo_bytes >> 4) << 16);
-}
-__device__ __forceinline__ void mma_ss_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "mov.b64 da, {%1, %3};\n\t"
-        "mov.b64 db, {%2, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mma_ts_lh(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "mov.b64 db, {%2, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(kDescHiSw128), "r"(idesc), "r"(accumulate) : "memory");
-}
 // Eight K steps (16 channels each) of D = A B^T in one statement, for K-major SWIZZLE_128B tiles whose
 // 128 channels lie in two 64-channel boxes `box16` (in 16-byte units) apart: A descriptors are passed
 // ready-made (they do not change while a CTA keeps its A tile), B is its first descriptor plus
@@ -263,10 +260,6 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-
-// Named barrier shared by two warps (64 threads): one warp arrives, the other waits.
-__device__ __forceinline__ void named_arrive64(uint32_t id) { asm volatile("bar.arrive %0, 64;" ::"r"(id) : "memory"); }
-__device__ __forceinline__ void named_sync64(uint32_t id) { asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory"); }
 
 // True in exactly one lane of a converged warp.
 __device__ __forceinline__ bool elect_one()
@@ -344,30 +337,6 @@ __device__ __forceinline__ float fmax3(float a, float b, float c)
     float r;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
     return r;
-}
-// 2^x for a pair of values on the FMA and integer pipes instead of the special-function unit:
-// x = floor(x) + f with f in [0,1) (the floor is taken by adding 1.5*2^23 with round-down, which
-// leaves it in the low mantissa bits), 2^f by a cubic with relative error below 1e-4 (fitted for
-// minimum maximum relative error with p(0) = 1), and the floor added to the exponent field.
-// Inputs are clamped at -126 so the result stays a normal number (about 1e-38 instead of 0).
-__device__ __forceinline__ float2 ex2_poly2(float2 x)
-{
-    const float kMagic = 12582912.f;                       // 1.5 * 2^23
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
-    unsigned long long xp, tp;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(xp) : "f"(x.x), "f"(x.y));
-    asm("{\n\t.reg .b64 m;\n\tmov.b64 m, {%1, %1};\n\tadd.rm.f32x2 %0, %2, m;\n\t}" : "=l"(tp) : "f"(kMagic), "l"(xp));
-    float2 t;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(t.x), "=f"(t.y) : "l"(tp));
-    const float2 fl = __fadd2_rn(t, make_float2(-kMagic, -kMagic));
-    const float2 f = __ffma2_rn(fl, make_float2(-1.f, -1.f), x);
-    float2 p = __ffma2_rn(f, make_float2(0.07706704f, 0.07706704f), make_float2(0.22764499f, 0.22764499f));
-    p = __ffma2_rn(p, f, make_float2(0.69511676f, 0.69511676f));
-    p = __ffma2_rn(p, f, make_float2(1.f, 1.f));
-    p.x = __int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23));
-    p.y = __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23));
-    return p;
 }
 // {hi, lo} -> packed bf16x2 with lo in bits 0-15 (round to nearest even)
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)

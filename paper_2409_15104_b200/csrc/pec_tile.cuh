@@ -14,21 +14,51 @@ struct TileJob {
     int32_t n_iv;
 };
 
-// Returns false when `tile` is past the last tile.  Packed batches walk cu_seqlens: request b
-// contributes ceil(len_b / block_m) tiles, each request starting a fresh tile.
+__device__ __forceinline__ void packed_job(int64_t req_start, int64_t pos0, int64_t req_len, int block_m, TileJob &job)
+{
+    job.q_row0 = req_start + pos0;
+    job.out_row0 = req_start + pos0;
+    job.q_pos0 = pos0;
+    job.n_rows = (int32_t)((req_len - pos0) < block_m ? (req_len - pos0) : block_m);
+    job.kv_row0 = req_start;
+    job.n_iv = 1;
+    job.iv_lo[0] = 0; job.iv_hi[0] = req_len;
+    job.iv_lo[1] = 0; job.iv_hi[1] = 0;
+}
+
+// Returns false when `tile` is past the last tile.  A single request's tiles run through its query
+// segments in ascending position, each segment starting a fresh tile.  Packed batches either read
+// entry `tile` of the work-list or walk cu_seqlens: request b contributes ceil(len_b / block_m)
+// tiles, each request starting a fresh tile.
 __device__ __forceinline__ bool locate_tile(const AttnParams &p, int64_t tile, int block_m, TileJob &job)
 {
     if (p.cu_seqlens == nullptr) {
-        const int64_t r0 = tile * block_m;
-        if (r0 >= p.chunk_len) return false;
-        job.q_row0 = p.chunk_start + r0;
-        job.out_row0 = r0;
-        job.q_pos0 = p.chunk_start + r0;
-        job.n_rows = (int32_t)((p.chunk_len - r0) < block_m ? (p.chunk_len - r0) : block_m);
-        job.kv_row0 = 0;
-        job.n_iv = p.n_iv;
-        job.iv_lo[0] = p.iv_lo[0]; job.iv_hi[0] = p.iv_hi[0];
-        job.iv_lo[1] = p.iv_lo[1]; job.iv_hi[1] = p.iv_hi[1];
+        int64_t t = tile;
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            if (s >= p.n_qseg) break;
+            const int64_t len = p.q_hi[s] - p.q_lo[s];
+            const int64_t nt = (len + block_m - 1) / block_m;
+            if (t < nt) {
+                const int64_t r0 = p.q_lo[s] + t * block_m;
+                job.q_row0 = r0;
+                job.out_row0 = r0 - p.out_pos0;
+                job.q_pos0 = r0;
+                job.n_rows = (int32_t)((p.q_hi[s] - r0) < block_m ? (p.q_hi[s] - r0) : block_m);
+                job.kv_row0 = 0;
+                job.n_iv = p.n_iv;
+                job.iv_lo[0] = p.iv_lo[0]; job.iv_hi[0] = p.iv_hi[0];
+                job.iv_lo[1] = p.iv_lo[1]; job.iv_hi[1] = p.iv_hi[1];
+                return true;
+            }
+            t -= nt;
+        }
+        return false;
+    }
+    if (p.worklist != nullptr) {
+        if (tile >= p.n_items) return false;
+        const int4 it = reinterpret_cast<const int4 *>(p.worklist)[tile];
+        packed_job(it.x, it.y, it.w, block_m, job);
         return true;
     }
     int64_t t = tile;
@@ -36,15 +66,7 @@ __device__ __forceinline__ bool locate_tile(const AttnParams &p, int64_t tile, i
         const int64_t s = p.cu_seqlens[b], e = p.cu_seqlens[b + 1];
         const int64_t nt = (e - s + block_m - 1) / block_m;
         if (t < nt) {
-            const int64_t r0 = t * block_m;
-            job.q_row0 = s + r0;
-            job.out_row0 = s + r0;
-            job.q_pos0 = r0;
-            job.n_rows = (int32_t)((e - s - r0) < block_m ? (e - s - r0) : block_m);
-            job.kv_row0 = s;
-            job.n_iv = 1;
-            job.iv_lo[0] = 0; job.iv_hi[0] = e - s;
-            job.iv_lo[1] = 0; job.iv_hi[1] = 0;
+            packed_job(s, t * block_m, e - s, block_m, job);
             return true;
         }
         t -= nt;
@@ -52,13 +74,13 @@ __device__ __forceinline__ bool locate_tile(const AttnParams &p, int64_t tile, i
     return false;
 }
 
-// The same search done by a whole converged warp: for a packed batch each lane takes every 32nd
-// request (the two table reads of all requests are in flight together instead of one dependent pair
-// per request), tile counts are prefix-summed with shuffles, and the lane that owns the tile's request
-// broadcasts it.  Every lane returns the same job.
+// The same search done by a whole converged warp: for a packed batch without a work-list each lane
+// takes every 32nd request (the two table reads of all requests are in flight together instead of
+// one dependent pair per request), tile counts are prefix-summed with shuffles, and the lane that
+// owns the tile's request broadcasts it.  Every lane returns the same job.
 __device__ __forceinline__ bool locate_tile_warp(const AttnParams &p, int64_t tile, int block_m, TileJob &job)
 {
-    if (p.cu_seqlens == nullptr) return locate_tile(p, tile, block_m, job);
+    if (p.cu_seqlens == nullptr || p.worklist != nullptr) return locate_tile(p, tile, block_m, job);
     const int lane = threadIdx.x & 31;
     int64_t before = 0;                                   // tiles of the requests in earlier groups of 32
     for (int b0 = 0; b0 < p.B; b0 += 32) {
@@ -78,15 +100,7 @@ __device__ __forceinline__ bool locate_tile_warp(const AttnParams &p, int64_t ti
             const int src = __ffs(who) - 1;
             const int64_t s_b = __shfl_sync(0xffffffffu, s, src), e_b = __shfl_sync(0xffffffffu, e, src);
             const int64_t first = __shfl_sync(0xffffffffu, before + incl - nt, src);
-            const int64_t r0 = (tile - first) * block_m;
-            job.q_row0 = s_b + r0;
-            job.out_row0 = s_b + r0;
-            job.q_pos0 = r0;
-            job.n_rows = (int32_t)((e_b - s_b - r0) < block_m ? (e_b - s_b - r0) : block_m);
-            job.kv_row0 = s_b;
-            job.n_iv = 1;
-            job.iv_lo[0] = 0; job.iv_hi[0] = e_b - s_b;
-            job.iv_lo[1] = 0; job.iv_hi[1] = 0;
+            packed_job(s_b, (tile - first) * block_m, e_b - s_b, block_m, job);
             return true;
         }
         before += __shfl_sync(0xffffffffu, incl, 31);

@@ -2,8 +2,10 @@
 
 Orchestration only (which call, which buffer): all arithmetic happens inside libpec.so.
 
-* partitioned_prefill - the per-step work of ring-attention sequence parallelism run as
-  virtual partitions on one GPU: plan, one partial per zigzag KV partition, running LSE merge.
+* PartitionedPrefill  - the per-step work of ring-attention sequence parallelism run as
+  virtual partitions on one GPU: plan, one launch per zigzag KV partition, each merging its
+  result into the running (O, LSE) state in its epilogue (or, chain=False, one partial per
+  partition and n-way LSE merge passes).
 * chunked_prefill     - a long prefill cut into preemptible chunks, each resumed from the
   stored K/V prefix (the pause points fall between kernel launches).
 * varlen_prefill      - a packed batch of short requests.
@@ -18,20 +20,25 @@ from . import binding
 
 
 class PartitionedPrefill:
-    """Buffers and call sequence for P virtual sequence partitions merged through their LSE.
+    """Buffers and call sequence for P virtual sequence partitions combined through their LSE.
 
-    Partials are kept in up to `max_live` fp32 buffers (bounded by `partial_budget_bytes`) and
-    merged with one n-way pass per group instead of P-1 two-way passes; with two buffers this
-    degenerates to the running two-way merge.
+    chain=True (default): one fp32 state; the launch of each partition merges its own result into
+    it in the attention epilogue (the online-softmax step across key segments), the last launch
+    writing the final output in the input dtype.  Partition 0 goes last because every row sees some
+    key of it, so the launch that rounds to the output dtype covers all rows.
+    chain=False: partials are kept in up to `max_live` fp32 buffers (bounded by
+    `partial_budget_bytes`) and merged with one n-way pass per group instead of P-1 two-way passes;
+    with two buffers this degenerates to the running two-way merge.
     """
 
-    def __init__(self, seq_len, hq, num_parts, dtype, device, part_align=128, partial_budget_bytes=80 << 30):
+    def __init__(self, seq_len, hq, num_parts, dtype, device, part_align=128, partial_budget_bytes=80 << 30, chain=True):
         self.S, self.Hq, self.P, self.align = seq_len, hq, num_parts, part_align
         self.dtype = dtype
+        self.chain = chain
         f32 = torch.float32
         per_partial = seq_len * hq * (128 * 4 + 4)
         self.max_live = max(2, min(num_parts, binding.PEC_MERGE_MAX_PARTS, partial_budget_bytes // max(per_partial, 1)))
-        n_buf = self.max_live if num_parts > 1 else 0
+        n_buf = 0 if num_parts == 1 else (1 if chain else self.max_live)
         self.part_o = [torch.empty((seq_len, hq, 128), dtype=f32, device=device) for _ in range(n_buf)]
         self.part_l = [torch.empty((seq_len, hq), dtype=f32, device=device) for _ in range(n_buf)]
         self.out_o = torch.empty((seq_len, hq, 128), dtype=dtype, device=device)
@@ -42,13 +49,14 @@ class PartitionedPrefill:
 
     def merge_launches(self):
         """Merge launches per step: the first group holds max_live partials, later ones max_live-1 new ones."""
-        if self.P == 1:
+        if self.P == 1 or self.chain:
             return 0
         rest = self.P - self.max_live
         return 1 + (0 if rest <= 0 else -(-rest // (self.max_live - 1)))
 
     def launches_per_step(self):
-        return self.P + self.merge_launches()
+        # chain: the first launch (partition 1) also fills the rows below that partition's first key
+        return self.P + (1 if self.chain and self.P > 1 else self.merge_launches())
 
     def run(self, q, k, v, stream=None, time_kernels=False, out=None):
         """Returns (o [S,Hq,128] in the input dtype, lse [S,Hq] fp32); `out` = (o, lse) buffers to write the
@@ -59,6 +67,13 @@ class PartitionedPrefill:
         self.merge_parts = []
         if P == 1:
             self._attn(q, k, v, 0, out_o, out_l, stream, time_kernels)
+            return out_o, out_l
+        if self.chain:
+            st_o, st_l = self.part_o[0], self.part_l[0]
+            self._attn(q, k, v, 1, st_o, st_l, stream, time_kernels)
+            for part in range(2, P):
+                self._attn(q, k, v, part, st_o, st_l, stream, time_kernels, acc=(st_o, st_l))
+            self._attn(q, k, v, 0, out_o, out_l, stream, time_kernels, acc=(st_o, st_l))
             return out_o, out_l
         p = 0
         first = True
@@ -99,10 +114,10 @@ class PartitionedPrefill:
         store.append(ev)
         return ev
 
-    def _attn(self, q, k, v, p, o, l, stream, time_kernels):
+    def _attn(self, q, k, v, p, o, l, stream, time_kernels, acc=None):
         ev = self._events(time_kernels, self.attn_events, stream)
         binding.pec_prefill_attn(q, k, v, seq_len=self.S, part_id=p, num_parts=self.P, part_align=self.align,
-                                 causal=True, o=o, lse=l, stream=stream)
+                                 causal=True, o=o, lse=l, stream=stream, acc=acc)
         if ev:
             ev[1].record(stream)
 
@@ -127,49 +142,47 @@ def chunked_prefill(q, k, v, chunk_len, o, lse, stream=None, between_chunks=None
     return plan["chunks"]
 
 
-def varlen_prefill(q, k, v, cu_seqlens, o=None, lse=None, stream=None):
-    """Packed batch of short causal prefills (cu_seqlens: int32 CUDA tensor [B+1])."""
-    return binding.pec_prefill_attn(q, k, v, cu_seqlens=cu_seqlens, causal=True, o=o, lse=lse, stream=stream)
+def make_worklist(cu_host, dtype, device):
+    """Heaviest-first tile list of a packed batch for the kernel that handles `dtype`, on the device
+    (cu_host: host sequence of B + 1 row offsets)."""
+    items = binding.pec_plan_worklist(cu_host, binding.pec_worklist_block_m(dtype), 128, True)
+    return torch.from_numpy(items).to(device, non_blocking=True)
+
+
+def varlen_prefill(q, k, v, cu_seqlens, o=None, lse=None, stream=None, worklist=None):
+    """Packed batch of short causal prefills (cu_seqlens: int32 CUDA tensor [B+1]; worklist: optional
+    tensor from make_worklist - without it every CTA searches cu_seqlens for its tile)."""
+    return binding.pec_prefill_attn(q, k, v, cu_seqlens=cu_seqlens, causal=True, o=o, lse=lse, stream=stream,
+                                    worklist=worklist)
 
 
 def ring_prefill(q, k, v, num_parts, part_align=128, stream=None):
     """The P x P (rank, ring step) launches of ring-attention SP (Section 2.2) on one GPU, no rank
     waiting for another: rank r owns the query rows of zigzag partition r and at step t attends to
-    the keys of partition (r - t) mod P; each rank merges its P partials through their LSE.
+    the keys of partition (r - t) mod P, one launch per (rank, step) that merges its result into the
+    rank's running (O, LSE) state.  Steps run t = 1, ..., P-1, 0: the rank's own keys come last because
+    every one of its rows sees some of them, so that launch can round the state to the output dtype.
     Returns (o [S,Hq,128] in the input dtype, lse [S,Hq] fp32, launches)."""
     S, Hq = q.shape[0], q.shape[1]
     P = num_parts
-    plan = binding.pec_plan_partitions(S, P, 0, part_align, 128, 128, True, tiles=False)
     f32 = torch.float32
     out_o = torch.empty((S, Hq, 128), dtype=q.dtype, device=q.device)
     out_l = torch.empty((S, Hq), dtype=f32, device=q.device)
-    longest = max((hi - lo for ivs in plan["parts"] for lo, hi in ivs), default=0)
-    run_o = torch.empty((max(longest, 1), Hq, 128), dtype=f32, device=q.device)
-    run_l = torch.empty((max(longest, 1), Hq), dtype=f32, device=q.device)
-    tmp_o, tmp_l = torch.empty_like(run_o), torch.empty_like(run_l)
+    if P == 1:
+        binding.pec_prefill_attn(q, k, v, seq_len=S, causal=True, o=out_o, lse=out_l, stream=stream)
+        return out_o, out_l, 1
+    st_o = torch.empty((S, Hq, 128), dtype=f32, device=q.device)    # every rank's state lives in its own rows
+    st_l = torch.empty((S, Hq), dtype=f32, device=q.device)
     launches = 0
     for r in range(P):
-        for lo, hi in plan["parts"][r]:
-            n = hi - lo
-            if n <= 0:
-                continue
-            for t in range(P):
-                first, last = t == 0, t == P - 1
-                direct = first and last                       # one rank: the partial is the result
-                o = out_o[lo:hi] if direct else (run_o[:n] if first else tmp_o[:n])
-                l = out_l[lo:hi] if direct else (run_l[:n] if first else tmp_l[:n])
-                binding.pec_prefill_attn(q, k, v, seq_len=S, chunk_start=lo, chunk_len=n, kv_len=S,
-                                         part_id=(r - t) % P, num_parts=P, part_align=part_align, causal=True,
-                                         o=o, lse=l, stream=stream)
-                launches += 1
-                if first:
-                    continue
-                if last:
-                    binding.pec_attn_merge(run_o[:n], run_l[:n], tmp_o[:n], tmp_l[:n], o_out=out_o[lo:hi],
-                                           lse_out=out_l[lo:hi], stream=stream)
-                else:
-                    binding.pec_attn_merge(run_o[:n], run_l[:n], tmp_o[:n], tmp_l[:n], inplace=True, stream=stream)
-                launches += 1
+        order = list(range(1, P)) + [0]
+        for i, t in enumerate(order):
+            first, last = i == 0, i == P - 1
+            binding.pec_prefill_attn(q, k, v, seq_len=S, part_id=(r - t) % P, num_parts=P, part_align=part_align,
+                                     q_part_id=r, q_num_parts=P, causal=True,
+                                     o=out_o if last else st_o, lse=out_l if last else st_l,
+                                     acc=None if first else (st_o, st_l), stream=stream)
+            launches += 1
     return out_o, out_l, launches
 
 

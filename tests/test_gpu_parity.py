@@ -352,9 +352,7 @@ def test_ring_prefill_every_rank_and_step_equals_monolithic(pec, S, P, hq, hkv):
     pec.check_status()
     want_o, want_l = oracle.prefill_attn(q, k, v, seq_len=S)
     compare(o, lse, want_o, want_l, *TOL[torch.bfloat16], f"ring S={S} P={P}")
-    # one attention launch per (rank interval, step) and one merge per step after the first
-    ivs = sum(1 for part in pec.pec_plan_partitions(S, P, 0, 64, 128, 128, True, tiles=False)["parts"] for lo, hi in part if hi > lo)
-    assert launches == ivs * (2 * P - 1)
+    assert launches == P * P                         # one launch per (rank, ring step), merges included
     # the plan's per-step work adds up to the causal total the launches computed
     assert sum(pec.pec_plan_ring(S, P, 64)["rank_total"]) == S * (S + 1) // 2
 
@@ -414,3 +412,129 @@ def test_streamed_prefill_matches_one_step_at_a_time(pec):
         assert torch.equal(o.cpu(), o_h) and torch.equal(l.cpu(), l_h), f"step {i}"
     want_o, want_l = oracle.prefill_attn(steps[-1][0], steps[-1][1], steps[-1][2], seq_len=S)
     compare(steps[-1][3], steps[-1][4], want_o, want_l, *TOL[torch.bfloat16], "streamed, last step")
+
+
+# ------------------------------------------------------------------ incoming state: online softmax across launches
+def _orders(P):
+    return {"ascending": list(range(P)), "descending": list(range(P - 1, -1, -1)),
+            "interleaved": list(range(1, P, 2)) + list(range(0, P, 2))}
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("S,P,align,order", [(1024, 4, 128, "ascending"), (700, 3, 64, "descending"), (515, 2, 1, "ascending"),
+                                             (130, 4, 128, "descending"), (2048, 8, 128, "interleaved"), (1500, 5, 32, "interleaved")])
+def test_chain_of_partition_launches_equals_monolithic(pec, dtype, S, P, align, order):
+    """Each launch merges its partition's result into the state the previous launches left (in place), the
+    last one writing the final output in the input dtype.  After every launch the state equals the oracle's
+    merge of the partials so far; at the end it equals the monolithic result."""
+    q, k, v = _qkv(17000 + S, S, 4, 2, dtype)
+    dq, dk, dv = _gpu(q, k, v)
+    seq = _orders(P)[order]
+    st_o = torch.full((S, 4, 128), float("nan"), dtype=torch.float32, device=DEV)
+    st_l = torch.full((S, 4), float("nan"), dtype=torch.float32, device=DEV)
+    want = None
+    for i, part in enumerate(seq[:-1]):
+        own = oracle.prefill_attn(q, k, v, seq_len=S, part_id=part, num_parts=P, part_align=align)
+        want = own if want is None else oracle.merge(*want, *own)
+        pec.pec_prefill_attn(dq, dk, dv, part_id=part, num_parts=P, part_align=align, o=st_o, lse=st_l,
+                             acc=None if i == 0 else (st_o, st_l))
+        pec.check_status()
+        compare(st_o, st_l, *want, *TOL[dtype], f"state after {i + 1} of {P} launches ({order})")
+    o, lse = pec.pec_prefill_attn(dq, dk, dv, part_id=seq[-1], num_parts=P, part_align=align, acc=(st_o, st_l), out_dtype=dtype)
+    pec.check_status()
+    assert o.dtype == dtype and o.data_ptr() != st_o.data_ptr()
+    compare(o, lse, *oracle.prefill_attn(q, k, v, seq_len=S), *TOL[dtype], f"chain of {P} launches ({order})")
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_incoming_state_with_empty_rows_on_either_side(pec, dtype):
+    """Rows empty in the state only, in the launch's own result only, in both, in neither; the incoming state's
+    buffers are separate from the outputs here and must come back unchanged."""
+    S, P = 1300, 4
+    q, k, v = _qkv(17100, S, 2, 1, dtype)
+    dq, dk, dv = _gpu(q, k, v)
+    # state: partition 2 over a short prefix (rows below 2b are empty); own: partition 3 (rows below 3b are empty)
+    a_o, a_l = pec.pec_prefill_attn(dq, dk, dv, part_id=2, num_parts=P, part_align=16, out_dtype=torch.float32)
+    keep_o, keep_l = a_o.clone(), a_l.clone()
+    want_a = oracle.prefill_attn(q, k, v, seq_len=S, part_id=2, num_parts=P, part_align=16)
+    want_b = oracle.prefill_attn(q, k, v, seq_len=S, part_id=3, num_parts=P, part_align=16)
+    assert np.isneginf(want_a[1]).any() and np.isneginf(want_b[1]).any()
+    for out in (torch.float32, dtype):
+        o, lse = pec.pec_prefill_attn(dq, dk, dv, part_id=3, num_parts=P, part_align=16, acc=(a_o, a_l), out_dtype=out)
+        pec.check_status()
+        compare(o, lse, *oracle.merge(*want_a, *want_b), *TOL[dtype], f"state + own, out {out}")
+        assert torch.equal(a_o, keep_o) and torch.equal(a_l, keep_l)
+    # the other way round: the state has keys where the launch has none
+    b_o, b_l = pec.pec_prefill_attn(dq, dk, dv, part_id=3, num_parts=P, part_align=16, out_dtype=torch.float32)
+    o, lse = pec.pec_prefill_attn(dq, dk, dv, part_id=0, num_parts=P, part_align=16, acc=(b_o, b_l), out_dtype=torch.float32)
+    pec.check_status()
+    compare(o, lse, *oracle.merge(*want_b, *oracle.prefill_attn(q, k, v, seq_len=S, part_id=0, num_parts=P, part_align=16)),
+            *TOL[dtype], "own + state")
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_chunk_partition_prefix_combinations_with_incoming_state(pec, seed):
+    """Two launches over different key partitions of a random chunk / prefix / alignment: the second takes the
+    first one's result as its incoming state, in place on even seeds, into a separate bf16 output on odd ones."""
+    c = _random_call(100 + seed)
+    if c["P"] == 1:
+        c["P"] = 3
+    c["part"] = c["part"] % c["P"]
+    other = (c["part"] + 1 + seed % (c["P"] - 1)) % c["P"]
+    q, k, v = _qkv(9300 + seed, c["S"], c["hq"], c["hkv"], torch.bfloat16)
+    kw = dict(seq_len=c["S"], chunk_start=c["c0"], chunk_len=c["n"], kv_len=c["kv_len"], num_parts=c["P"],
+              part_align=c["align"], causal=c["causal"])
+    want = oracle.merge(*oracle.prefill_attn(q, k, v, part_id=c["part"], **kw), *oracle.prefill_attn(q, k, v, part_id=other, **kw))
+    dq, dk, dv = _gpu(q, k, v)
+    dk[c["kv_len"]:] = float("nan"); dv[c["kv_len"]:] = float("nan")
+    st_o, st_l = pec.pec_prefill_attn(dq, dk, dv, part_id=c["part"], out_dtype=torch.float32, **kw)
+    if seed % 2 == 0:
+        o, lse = pec.pec_prefill_attn(dq, dk, dv, part_id=other, o=st_o, lse=st_l, acc=(st_o, st_l), **kw)
+    else:
+        o, lse = pec.pec_prefill_attn(dq, dk, dv, part_id=other, acc=(st_o, st_l), out_dtype=torch.bfloat16, **kw)
+    pec.check_status()
+    compare(o, lse, *want, *TOL[torch.bfloat16], f"random call with state {c} + partition {other}")
+
+
+# ------------------------------------------------------------------ a ring rank's rows in one launch
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("S,P,align,c0,n", [(1024, 4, 128, 0, 1024), (1500, 3, 64, 0, 1500), (900, 2, 1, 100, 700), (300, 8, 16, 0, 300)])
+def test_query_partition_launch_touches_only_its_rows(pec, dtype, S, P, align, c0, n):
+    q, k, v = _qkv(18000 + S, S, 4, 2, dtype)
+    dq, dk, dv = _gpu(q, k, v)
+    for r in range(P):
+        rows = oracle.partition_rows(S, P, r, align, c0, n)
+        for s in {(r - 1) % P, r, (r + 1) % P}:
+            o = torch.full((n, 4, 128), 7.0, dtype=torch.float32, device=DEV)
+            lse = torch.full((n, 4), 7.0, dtype=torch.float32, device=DEV)
+            pec.pec_prefill_attn(dq, dk, dv, seq_len=S, chunk_start=c0, chunk_len=n, kv_len=S, part_id=s, num_parts=P,
+                                 part_align=align, q_part_id=r, q_num_parts=P, o=o, lse=lse)
+            pec.check_status()
+            mine = torch.zeros(n, dtype=torch.bool)
+            if rows:
+                idx = torch.as_tensor(rows) - c0
+                mine[idx] = True
+                want = oracle.prefill_attn(q, k, v, seq_len=S, chunk_start=c0, chunk_len=n, kv_len=S, part_id=s, num_parts=P,
+                                           part_align=align, rows=rows)
+                compare(o[idx.to(DEV)], lse[idx.to(DEV)], *want, *TOL[dtype], f"rank {r} rows x keys of {s}")
+            assert (o.cpu()[~mine] == 7).all() and (lse.cpu()[~mine] == 7).all(), "rows of other ranks were written"
+
+
+# ------------------------------------------------------------------ packed batch through a work-list
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("lens", [[5], [1, 300, 0, 77, 129, 64], [700, 20, 1200, 256, 257], [(i * 37) % 200 for i in range(70)]],
+                         ids=["one", "with_empty", "mixed", "seventy"])
+def test_varlen_batch_through_a_worklist(pec, dtype, lens):
+    from paper_2409_15104_b200 import prefill
+    cu = workloads.cu_seqlens(lens)
+    T = cu[-1]
+    q, k, v = _qkv(19000 + T, T, 4, 2, dtype)
+    dq, dk, dv = _gpu(q, k, v)
+    dcu = torch.tensor(cu, dtype=torch.int32, device=DEV)
+    wl = prefill.make_worklist(cu, dtype, DEV)
+    assert wl.shape == (sum(-(-n // pec.pec_worklist_block_m(dtype)) for n in lens), 4)
+    o, lse = prefill.varlen_prefill(dq, dk, dv, dcu, worklist=wl)
+    o2, lse2 = prefill.varlen_prefill(dq, dk, dv, dcu)
+    pec.check_status()
+    compare(o, lse, *oracle.varlen_attn(q, k, v, cu), *TOL[dtype], f"varlen work-list {lens[:6]}")
+    assert torch.equal(o, o2) and torch.equal(lse, lse2)          # same tiles, another order
