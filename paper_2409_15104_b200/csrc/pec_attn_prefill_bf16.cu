@@ -425,17 +425,31 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         // Each warp instead stages 32 rows x 256 bytes in its quarter of the stage's Q tile (no longer
         // read once the stage's last product is done; 16-byte chunks XOR-swizzled by row against bank
         // conflicts) and writes it out two rows per instruction, 256 contiguous bytes each.
+        const bool has_acc = p.acc_o != nullptr;
+        const int sub = lane >> 4, chunk = lane & 15;                            // read-back: row parity and 16-byte chunk
+        // The incoming state's LSE and its first 64 channels are asked for before the wait for the last product,
+        // so that their latency runs under it (the lines were prefetched towards the L2 one tile ago).
+        const float *acc_base = has_acc ? p.acc_o + ((row0 + sub) * p.Hq + h) * kHeadDim + chunk * 4 : nullptr;
+        float la = -INFINITY;
+        float4 inc[16];
+        if (has_acc && sh->g.rows[st] > 0) {
+            if (lane < rows_valid) la = p.acc_lse[(row0 + lane) * p.Hq + h];
+            const float *src = acc_base;
+#pragma unroll
+            for (int rr = 0; rr < 16; ++rr, src += 2 * (int64_t)p.Hq * kHeadDim) {
+                inc[rr] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (2 * rr + sub < rows_valid) inc[rr] = *reinterpret_cast<const float4 *>(src);
+            }
+        }
         if (ok && n_hf > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->o_final[st]), 0, sh, p));
         // A stage without keys never waited for its Q tile: the load must have landed before the tile is reused.
         if (ok && n_hf == 0 && n_max > 0) ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->bar_q[st]), 0, sh, p));
         if (ok && sh->g.rows[st] > 0) {
             tc_fence_after();
-            const bool has_acc = p.acc_o != nullptr;
             const bool empty = (l_run == 0.f);
             float c_own = empty ? 0.f : 1.f / l_run, c_acc = 0.f;
             float lse_row = empty ? -INFINITY : m_ref * 0.6931471805599453f + logf(l_run);
             if (has_acc) {
-                const float la = lane < rows_valid ? p.acc_lse[(row0 + lane) * p.Hq + h] : -INFINITY;
                 const float mx = fmaxf(lse_row, la);
                 if (mx != -INFINITY) {
                     const float e_own = empty ? 0.f : expf(lse_row - mx), e_acc = (la == -INFINITY) ? 0.f : expf(la - mx);
@@ -450,7 +464,6 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             const bool skip = in_place && __all_sync(0xffffffffu, empty || lane >= rows_valid);
             uint8_t *stage_buf = smem_raw + (tiles - raw) + st * kTileBytes + quarter * 8192;
             uint8_t *my_row = stage_buf + lane * 256;
-            const int sub = lane >> 4, chunk = lane & 15;                        // read-back: row parity and 16-byte chunk
             const int o_esz = p.o_is_bf16 ? 2 : 4;
             const int64_t row_bytes = (int64_t)p.Hq * kHeadDim * o_esz;
             uint8_t *out = static_cast<uint8_t *>(p.o) + (row0 + sub) * row_bytes + (int64_t)h * kHeadDim * o_esz;
@@ -491,13 +504,11 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     if (2 * rr + sub < rows_valid) *reinterpret_cast<uint4 *>(dst) = val[rr];
             } else {
                 // Two passes of 64 channels staged as fp32 (256 bytes of a row each).
-                const float *acc_base = has_acc ? p.acc_o + ((row0 + sub) * p.Hq + h) * kHeadDim + chunk * 4 : nullptr;
 #pragma unroll 1
                 for (int pass = 0; pass < 2; ++pass) {
-                    // The incoming state's loads go first: their latency runs under the TMEM read and the staging.
-                    float4 inc[16];
-                    if (has_acc) {
-                        const float *src = acc_base + pass * 64;
+                    // The second half of the incoming state: its latency runs under the TMEM read and the staging.
+                    if (has_acc && pass == 1) {
+                        const float *src = acc_base + 64;
 #pragma unroll
                         for (int rr = 0; rr < 16; ++rr, src += 2 * (int64_t)p.Hq * kHeadDim) {
                             inc[rr] = make_float4(0.f, 0.f, 0.f, 0.f);

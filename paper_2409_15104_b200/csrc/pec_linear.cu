@@ -187,9 +187,11 @@ extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_
     }
     const int64_t pairs = (M + 2 * lin::kBM - 1) / (2 * lin::kBM), gn = (N + lin::kBN - 1) / lin::kBN;
     if (gn > 65535) { set_error("pec_linear: N too large"); return PEC_ERR_UNSUPPORTED; }
-    // Rows of x per band: what leaves room for w in about 96 MB of the L2 (at least 4 row pairs, at most 32).
-    const int64_t w_bytes = (int64_t)N * K * 2, pair_bytes = (int64_t)2 * lin::kBM * K * 2;
-    int64_t band = ((int64_t)96 << 20) > w_bytes ? (((int64_t)96 << 20) - w_bytes) / pair_bytes : 0;
+    // Rows of x per band: about 24 MB of x (at least 4 row pairs, at most 32).  Measured on [32768, 4096] x
+    // [6144, 4096]^T: bands of 12 row pairs (24 MB) 1409 TFLOP/s, 4: 1382, 8: 1404, 16: 1401, 23: 1385, 32: 1348 -
+    // the L2 serves both dies and also carries w and the stream of y, so far less than its 126 MB holds a band.
+    const int64_t pair_bytes = (int64_t)2 * lin::kBM * K * 2;
+    int64_t band = ((int64_t)24 << 20) / pair_bytes;
     band = band < 4 ? 4 : (band > 32 ? 32 : band);
     dim3 grid((unsigned)(2 * pairs), (unsigned)gn);           // clusters of two CTAs along x
     lin::linear_kernel<<<grid, lin::kThreads, lin::kSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(
