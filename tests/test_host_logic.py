@@ -88,6 +88,16 @@ def _args(**over):
     (dict(q=4100), -3), (dict(k_stride_t=8 * 128 + 4), -3), (dict(q_stride_h=64), -1),
     (dict(cu_seqlens=4096, B=2, chunk_len=100), -1), (dict(softmax_scale=float("nan")), -1),
     (dict(part_align=0), -1),
+    (dict(acc_o=8192), -1),                                            # incoming state without its LSE
+    (dict(acc_o=4096, acc_lse=8192, o_dtype=binding.PEC_F32), -1),    # o is the state's buffer, lse is not
+    (dict(acc_o=4096, acc_lse=4096), -1),                              # in-place merge needs fp32 output
+    (dict(acc_o=8196, acc_lse=12288), -3),
+    (dict(q_num_parts=4, q_part_id=4), -1), (dict(q_num_parts=2, q_part_id=-1), -1),
+    (dict(cu_seqlens=4096, B=2, q_num_parts=2), -1),                   # query partitions are for single requests
+    (dict(status=None), -1),                                           # bf16 inputs need the status word
+    (dict(worklist=4096, n_items=3), -1),                              # a work-list without cu_seqlens
+    (dict(cu_seqlens=4096, B=2, worklist=4096, n_items=3, worklist_block_m=64), -1),   # built for the other kernel's tiles
+    (dict(cu_seqlens=4096, B=2, worklist=4100, n_items=3, worklist_block_m=256), -1),
 ])
 def test_prefill_attn_validates_on_the_host(over, code):
     lib = binding.load()
