@@ -47,7 +47,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Wa
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 2)
 linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-                   __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t band, int32_t *status,
+                   __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t band, int32_t by_cols, int32_t *status,
               long long wait_cycles, int32_t test_skip_last_load)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -58,15 +58,29 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
     const uint32_t rank = cluster_ctarank();                  // 0 = leader
     // Tile order.  Clusters are dispatched x-fastest; taken as they come (all row pairs of one column
     // of y, then the next column) every column would stream the whole of x from HBM again.  The
-    // dispatch index is re-read as bands of `band` row pairs: within a band the row pairs vary fastest
-    // and the columns next, so a band's rows of x (and all of w) stay in L2 while its columns are done.
+    // dispatch index is re-read in bands.  by_cols == 0: bands of `band` row pairs, within a band the row
+    // pairs vary fastest and the columns next, so a band's rows of x stay in L2 while its columns are done
+    // (x is read once, w once per band).  by_cols == 1: bands of `band` columns of y, within a band the
+    // columns vary fastest and the row pairs next (w is read once, x once per band).  The host picks the
+    // cheaper of the two.
     const int pairs = (int)(gridDim.x >> 1), gn = (int)gridDim.y;
     const int64_t seq = (int64_t)blockIdx.y * pairs + (blockIdx.x >> 1);
-    const int band_i = (int)(seq / ((int64_t)band * gn));
-    const int band_pairs = (pairs - band_i * band) < band ? (pairs - band_i * band) : band;
-    const int within = (int)(seq - (int64_t)band_i * band * gn);
-    const int64_t m0 = (int64_t)(band_i * band + within % band_pairs) * (2 * kBM) + rank * kBM;
-    const int n0 = (within / band_pairs) * kBN;
+    int pair_i, col_i;
+    if (!by_cols) {
+        const int band_i = (int)(seq / ((int64_t)band * gn));
+        const int band_pairs = (pairs - band_i * band) < band ? (pairs - band_i * band) : band;
+        const int within = (int)(seq - (int64_t)band_i * band * gn);
+        pair_i = band_i * band + within % band_pairs;
+        col_i = within / band_pairs;
+    } else {
+        const int band_i = (int)(seq / ((int64_t)band * pairs));
+        const int band_cols = (gn - band_i * band) < band ? (gn - band_i * band) : band;
+        const int within = (int)(seq - (int64_t)band_i * band * pairs);
+        col_i = band_i * band + within % band_cols;
+        pair_i = within / band_cols;
+    }
+    const int64_t m0 = (int64_t)pair_i * (2 * kBM) + rank * kBM;
+    const int n0 = col_i * kBN;
     const int n_kb = (K + kBK - 1) / kBK;
     const WaitCtx wctx = {&sh->abort_flag, status, wait_cycles};
 
@@ -187,15 +201,20 @@ extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_
     }
     const int64_t pairs = (M + 2 * lin::kBM - 1) / (2 * lin::kBM), gn = (N + lin::kBN - 1) / lin::kBN;
     if (gn > 65535) { set_error("pec_linear: N too large"); return PEC_ERR_UNSUPPORTED; }
-    // Rows of x per band: about 24 MB of x (at least 4 row pairs, at most 32).  Measured on [32768, 4096] x
-    // [6144, 4096]^T: bands of 12 row pairs (24 MB) 1409 TFLOP/s, 4: 1382, 8: 1404, 16: 1401, 23: 1385, 32: 1348 -
-    // the L2 serves both dies and also carries w and the stream of y, so far less than its 126 MB holds a band.
-    const int64_t pair_bytes = (int64_t)2 * lin::kBM * K * 2;
-    int64_t band = ((int64_t)24 << 20) / pair_bytes;
+    // Bands of about 24 MB of one operand (4 to 32 tiles).  Measured on [32768, 4096] x [6144, 4096]^T with bands of
+    // row pairs: 12 (24 MB) 1409 TFLOP/s, 4: 1382, 8: 1404, 16: 1401, 23: 1385, 32: 1348 - the L2 serves both dies and
+    // also carries the other operand and the stream of y, so far less than its 126 MB holds a band.  Bands of x
+    // rows read x once and w once per band; bands of w rows (columns of y) the other way round: take the cheaper.
+    const int64_t tile_bytes = (int64_t)2 * lin::kBM * K * 2;           // 256 rows of either operand
+    int64_t band = ((int64_t)24 << 20) / tile_bytes;
     band = band < 4 ? 4 : (band > 32 ? 32 : band);
+    const int64_t x_bytes = (int64_t)M * K * 2, w_bytes = (int64_t)N * K * 2;
+    const int64_t by_rows_traffic = x_bytes + w_bytes * ((pairs + band - 1) / band);
+    const int64_t by_cols_traffic = w_bytes + x_bytes * ((gn + band - 1) / band);
+    const int32_t by_cols = by_cols_traffic < by_rows_traffic ? 1 : 0;
     dim3 grid((unsigned)(2 * pairs), (unsigned)gn);           // clusters of two CTAs along x
     lin::linear_kernel<<<grid, lin::kThreads, lin::kSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(
-        tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, (int32_t)band, status,
+        tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, (int32_t)band, by_cols, status,
         (long long)wait_limit_cycles(), test_skip_last_load());
     const cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("pec_linear: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
