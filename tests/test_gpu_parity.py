@@ -538,3 +538,27 @@ def test_varlen_batch_through_a_worklist(pec, dtype, lens):
     pec.check_status()
     compare(o, lse, *oracle.varlen_attn(q, k, v, cu), *TOL[dtype], f"varlen work-list {lens[:6]}")
     assert torch.equal(o, o2) and torch.equal(lse, lse2)          # same tiles, another order
+
+
+# ------------------------------------------------------------------ the two ways a partitioned step combines its partitions
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("budget_parts", [2, 3, 16])
+def test_partitioned_prefill_by_merge_passes_equals_the_chained_form(pec, dtype, budget_parts):
+    """chain=False keeps partials and merges them n at a time (2: the running two-way merge; 3: several n-way
+    groups; 16: one pass); chain=True merges in the attention epilogue.  Both against the oracle."""
+    from paper_2409_15104_b200.prefill import PartitionedPrefill
+    S, hq, hkv, P = 1536, 4, 2, 6
+    q, k, v = _qkv(20000 + budget_parts, S, hq, hkv, dtype)
+    dq, dk, dv = _gpu(q, k, v)
+    want = oracle.prefill_attn(q, k, v, seq_len=S)
+    per_partial = S * hq * (128 * 4 + 4)
+    merged = PartitionedPrefill(S, hq, P, dtype, DEV, part_align=64, partial_budget_bytes=budget_parts * per_partial, chain=False)
+    assert merged.max_live == min(budget_parts, P)
+    o, lse = merged.run(dq, dk, dv)
+    pec.check_status()
+    compare(o, lse, *want, *TOL[dtype], f"merge passes, {merged.max_live} partials live")
+    assert len(merged.merge_parts) == merged.merge_launches()
+    chained = PartitionedPrefill(S, hq, P, dtype, DEV, part_align=64)
+    o2, lse2 = chained.run(dq, dk, dv)
+    pec.check_status()
+    compare(o2, lse2, *want, *TOL[dtype], "chained")
