@@ -92,6 +92,14 @@ enum { PEC_TILE_SKIP = 0, PEC_TILE_PARTIAL = 1, PEC_TILE_FULL = 2 };
  * pass.  o / lse may be the very buffers acc_o / acc_lse (both, o_dtype PEC_F32): rows that see no key
  * of this call's subset then stay untouched.  Only the last call of a chain should round to PEC_BF16.
  *
+ * overlap_previous = 1 tells the library that q, k and v (and cu_seqlens / worklist) were complete before the kernel
+ * that precedes this call on the stream was enqueued - true for every launch but the first of a chain over the key
+ * partitions, or of a ring rank's steps.  The bf16 kernel may then start on SMs that the preceding kernel has already
+ * left (programmatic dependent launch) and work through its key tiles while that kernel's last CTAs finish; it still
+ * waits for the preceding kernel to complete before it reads the incoming state or writes o / lse.  Chains of short
+ * launches lose their launch gaps and partial last waves that way.  With 0 (default) the call is ordered after
+ * everything enqueued before it, as any kernel is.
+ *
  * Packed batches may pass a work-list (worklist, n_items, worklist_block_m) made by pec_plan_worklist
  * and copied to the device by the caller: tiles then run heaviest first across requests and no CTA
  * searches cu_seqlens.  worklist_block_m must equal pec_worklist_block_m(in_dtype).
@@ -129,6 +137,7 @@ typedef struct {
     const int32_t *worklist;    /* device; [n_items][4] from pec_plan_worklist, or NULL  */
     int32_t n_items;
     int32_t worklist_block_m;
+    int32_t overlap_previous;   /* 0 or 1, see above                                     */
 } pec_attn_args;
 
 /*

@@ -49,6 +49,7 @@ class pec_attn_args(ctypes.Structure):
         ("acc_o", ctypes.c_void_p), ("acc_lse", ctypes.c_void_p),
         ("q_part_id", ctypes.c_int32), ("q_num_parts", ctypes.c_int32),
         ("worklist", ctypes.c_void_p), ("n_items", ctypes.c_int32), ("worklist_block_m", ctypes.c_int32),
+        ("overlap_previous", ctypes.c_int32),
     ]
 
 
@@ -198,7 +199,7 @@ def check_status(device=None):
 def pec_prefill_attn(q, k, v, *, seq_len=None, chunk_start=0, chunk_len=None, kv_len=None,
                      part_id=0, num_parts=1, part_align=128, causal=True, softmax_scale=0.0,
                      cu_seqlens=None, out_dtype=None, o=None, lse=None, stream=None,
-                     acc=None, q_part_id=0, q_num_parts=0, worklist=None):
+                     acc=None, q_part_id=0, q_num_parts=0, worklist=None, overlap_previous=False):
     """Partial attention of one chunk / partition / packed batch; returns (o, lse).
 
     q [T, Hq, 128], k / v [Tk, Hkv, 128] CUDA tensors (last dim contiguous).  Single request:
@@ -208,7 +209,8 @@ def pec_prefill_attn(q, k, v, *, seq_len=None, chunk_start=0, chunk_len=None, kv
     acc = (o, lse) fp32 tensors: an incoming state of the same rows that the call merges its result
     into (pass the same tensors as o / lse for an in-place chain).  q_num_parts > 1 restricts the
     query rows to zigzag partition q_part_id.  worklist: int32 CUDA tensor [n, 4] from
-    pec_plan_worklist (packed batches).
+    pec_plan_worklist (packed batches).  overlap_previous=True: the inputs were complete before the kernel that
+    precedes this call on the stream, so the call may start while that kernel's last CTAs finish.
     """
     lib = load()
     assert q.is_cuda and k.is_cuda and v.is_cuda
@@ -253,6 +255,7 @@ def pec_prefill_attn(q, k, v, *, seq_len=None, chunk_start=0, chunk_len=None, kv
         assert acc_o.shape == (chunk_len, Hq, D) and acc_l.shape == (chunk_len, Hq)
         a.acc_o, a.acc_lse = acc_o.data_ptr(), acc_l.data_ptr()
     a.q_part_id, a.q_num_parts = q_part_id, q_num_parts
+    a.overlap_previous = 1 if overlap_previous else 0
     if worklist is not None:
         assert worklist.is_cuda and worklist.dtype == torch.int32 and worklist.is_contiguous()
         a.worklist, a.n_items = worklist.data_ptr(), worklist.shape[0]

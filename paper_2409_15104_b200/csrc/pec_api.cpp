@@ -84,6 +84,7 @@ static int resolve(const pec_attn_args *a, AttnParams &p)
         set_error("pec_prefill_attn: need 0 <= q_part_id < q_num_parts, single request only");
         return PEC_ERR_INVALID_ARG;
     }
+    if (a->overlap_previous != 0 && a->overlap_previous != 1) { set_error("pec_prefill_attn: overlap_previous must be 0 or 1"); return PEC_ERR_INVALID_ARG; }
     if (a->in_dtype == PEC_BF16 && !a->status) { set_error("pec_prefill_attn: bf16 inputs need a status word"); return PEC_ERR_INVALID_ARG; }
     if (a->worklist) {
         if (!a->cu_seqlens || a->n_items < 0 || (reinterpret_cast<uintptr_t>(a->worklist) & 15u)) {
@@ -129,6 +130,7 @@ static int resolve(const pec_attn_args *a, AttnParams &p)
     p.total_rows = a->chunk_len;
     p.out_pos0 = a->chunk_start;
     p.acc_o = a->acc_o; p.acc_lse = a->acc_lse;
+    p.overlap_previous = a->overlap_previous;
     p.wait_cycles = wait_limit_cycles();
     p.test_skip_last_load = test_skip_last_load();
     // Query rows: the chunk, or its intersection with the two blocks of zigzag partition q_part_id.

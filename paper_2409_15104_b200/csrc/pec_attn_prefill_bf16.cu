@@ -164,6 +164,9 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             }
         }
     } else if (tid == 32) {
+        // Every CTA of the grid has started once the last one has said so: from then on a following launch that
+        // may overlap this one (overlap_previous) takes the SMs this grid leaves.
+        griddep_launch_dependents();
         prefetch_tmap(&tm_q); prefetch_tmap(&tm_k); prefetch_tmap(&tm_v);
         for (int st = 0; st < 2; ++st) {
             mbar_init(smem_u32(&sh->s_full[st]), 1);
@@ -425,6 +428,9 @@ attn_prefill_bf16_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         // Each warp instead stages 32 rows x 256 bytes in its quarter of the stage's Q tile (no longer
         // read once the stage's last product is done; 16-byte chunks XOR-swizzled by row against bank
         // conflicts) and writes it out two rows per instruction, 256 contiguous bytes each.
+        // A launch that overlaps its predecessor has walked its key tiles beside that kernel's last CTAs; the incoming
+        // state and the output buffers are the predecessor's (or an earlier kernel's) until it has completed.
+        griddep_wait();
         const bool has_acc = p.acc_o != nullptr;
         const int sub = lane >> 4, chunk = lane & 15;                            // read-back: row parity and 16-byte chunk
         // The incoming state's LSE and its first 64 channels are asked for before the wait for the last product,
@@ -615,9 +621,18 @@ int launch_attn_prefill_bf16(const AttnParams &p, cudaStream_t stream)
         return PEC_ERR_CUDA;
     }
     if (tiles > 0x7fffffff || p.Hq > 65535) { set_error("pec_prefill_attn: grid too large"); return PEC_ERR_UNSUPPORTED; }
-    dim3 grid((unsigned)tiles, (unsigned)p.Hq, 1);
-    attn_prefill_bf16_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_q, tm_k, tm_v, p);
-    const cudaError_t err = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)tiles, (unsigned)p.Hq, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = p.overlap_previous ? 1 : 0;
+    cudaError_t err = cudaLaunchKernelEx(&cfg, attn_prefill_bf16_kernel, tm_q, tm_k, tm_v, p);
+    if (err == cudaSuccess) err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("pec_prefill_attn: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;
 }

@@ -42,6 +42,7 @@ struct AttnParams {
     float scale;                     // softmax scale
     float scale_log2;                // scale * log2(e)
     int32_t o_is_bf16;
+    int32_t overlap_previous;        // launch as a programmatic dependent of the preceding kernel on the stream
     int32_t *status;
     int64_t wait_cycles;             // limit of every device-side barrier wait, in SM clock cycles
     int32_t test_skip_last_load;     // test hook: the loader leaves out its last item (a wait must then run out)

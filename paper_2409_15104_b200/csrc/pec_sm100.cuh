@@ -75,6 +75,13 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     return true;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// launch_dependents: once every CTA of this grid has executed it (or exited), a following kernel that was launched
+// as a programmatic dependent may start on SMs this grid no longer needs.  wait: blocks until the kernel(s) this grid
+// depends on have completed and their memory is visible; a no-op in a grid that was launched the ordinary way.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- TMA
 // 3-D tiled load: coordinates are (innermost, middle, outermost) in elements.
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, uint32_t bar, int c0, int c1, int c2)

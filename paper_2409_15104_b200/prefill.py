@@ -60,7 +60,8 @@ class PartitionedPrefill:
 
     def run(self, q, k, v, stream=None, time_kernels=False, out=None):
         """Returns (o [S,Hq,128] in the input dtype, lse [S,Hq] fp32); `out` = (o, lse) buffers to write the
-        result to instead of the runner's own."""
+        result to instead of the runner's own.  time_kernels=True brackets every launch with CUDA events and, so
+        that those mean something, lets no launch start before its predecessor has finished."""
         P = self.P
         out_o, out_l = (self.out_o, self.out_l) if out is None else out
         self.plan = binding.pec_plan_partitions(self.S, P, 0, self.align, 128, 128, True, tiles=False)
@@ -71,9 +72,11 @@ class PartitionedPrefill:
         if self.chain:
             st_o, st_l = self.part_o[0], self.part_l[0]
             self._attn(q, k, v, 1, st_o, st_l, stream, time_kernels)
+            # q, k, v were there before the first launch: every later launch of the chain may start on the SMs its
+            # predecessor has left (it waits for that launch before it touches the state)
             for part in range(2, P):
-                self._attn(q, k, v, part, st_o, st_l, stream, time_kernels, acc=(st_o, st_l))
-            self._attn(q, k, v, 0, out_o, out_l, stream, time_kernels, acc=(st_o, st_l))
+                self._attn(q, k, v, part, st_o, st_l, stream, time_kernels, acc=(st_o, st_l), overlap=not time_kernels)
+            self._attn(q, k, v, 0, out_o, out_l, stream, time_kernels, acc=(st_o, st_l), overlap=not time_kernels)
             return out_o, out_l
         p = 0
         first = True
@@ -114,10 +117,10 @@ class PartitionedPrefill:
         store.append(ev)
         return ev
 
-    def _attn(self, q, k, v, p, o, l, stream, time_kernels, acc=None):
+    def _attn(self, q, k, v, p, o, l, stream, time_kernels, acc=None, overlap=False):
         ev = self._events(time_kernels, self.attn_events, stream)
         binding.pec_prefill_attn(q, k, v, seq_len=self.S, part_id=p, num_parts=self.P, part_align=self.align,
-                                 causal=True, o=o, lse=l, stream=stream, acc=acc)
+                                 causal=True, o=o, lse=l, stream=stream, acc=acc, overlap_previous=overlap)
         if ev:
             ev[1].record(stream)
 
@@ -178,10 +181,11 @@ def ring_prefill(q, k, v, num_parts, part_align=128, stream=None):
         order = list(range(1, P)) + [0]
         for i, t in enumerate(order):
             first, last = i == 0, i == P - 1
+            # every launch after the very first may overlap its predecessor: the inputs were there before either
             binding.pec_prefill_attn(q, k, v, seq_len=S, part_id=(r - t) % P, num_parts=P, part_align=part_align,
                                      q_part_id=r, q_num_parts=P, causal=True,
                                      o=out_o if last else st_o, lse=out_l if last else st_l,
-                                     acc=None if first else (st_o, st_l), stream=stream)
+                                     acc=None if first else (st_o, st_l), stream=stream, overlap_previous=launches > 0)
             launches += 1
     return out_o, out_l, launches
 

@@ -562,3 +562,29 @@ def test_partitioned_prefill_by_merge_passes_equals_the_chained_form(pec, dtype,
     o2, lse2 = chained.run(dq, dk, dv)
     pec.check_status()
     compare(o2, lse2, *want, *TOL[dtype], "chained")
+
+
+def test_launches_that_overlap_their_predecessor_give_the_same_bits(pec):
+    """overlap_previous lets a launch start on the SMs its predecessor has left; it must still see the complete
+    incoming state.  A chain of short launches (many more CTAs than SMs, state merged in place) run both ways,
+    several times over, gives identical bits; the chain equals the monolithic oracle result."""
+    S, hq, hkv, P = 4096, 16, 4, 8
+    q, k, v = _qkv(22000, S, hq, hkv, torch.bfloat16)
+    dq, dk, dv = _gpu(q, k, v)
+
+    def chain(overlap):
+        st_o = torch.full((S, hq, 128), float("nan"), dtype=torch.float32, device=DEV)
+        st_l = torch.full((S, hq), float("nan"), dtype=torch.float32, device=DEV)
+        pec.pec_prefill_attn(dq, dk, dv, part_id=1, num_parts=P, o=st_o, lse=st_l)
+        for part in range(2, P):
+            pec.pec_prefill_attn(dq, dk, dv, part_id=part, num_parts=P, o=st_o, lse=st_l, acc=(st_o, st_l), overlap_previous=overlap)
+        return pec.pec_prefill_attn(dq, dk, dv, part_id=0, num_parts=P, acc=(st_o, st_l), out_dtype=torch.bfloat16,
+                                    overlap_previous=overlap)
+
+    base = chain(False)
+    pec.check_status()
+    for _ in range(5):
+        o, lse = chain(True)
+        pec.check_status()
+        assert torch.equal(o, base[0]) and torch.equal(lse, base[1])
+    compare(o, lse, *oracle.prefill_attn(q, k, v, seq_len=S), *TOL[torch.bfloat16], "overlapping chain")

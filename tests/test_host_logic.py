@@ -95,6 +95,7 @@ def _args(**over):
     (dict(q_num_parts=4, q_part_id=4), -1), (dict(q_num_parts=2, q_part_id=-1), -1),
     (dict(cu_seqlens=4096, B=2, q_num_parts=2), -1),                   # query partitions are for single requests
     (dict(status=None), -1),                                           # bf16 inputs need the status word
+    (dict(overlap_previous=2), -1),
     (dict(worklist=4096, n_items=3), -1),                              # a work-list without cu_seqlens
     (dict(cu_seqlens=4096, B=2, worklist=4096, n_items=3, worklist_block_m=64), -1),   # built for the other kernel's tiles
     (dict(cu_seqlens=4096, B=2, worklist=4100, n_items=3, worklist_block_m=256), -1),
