@@ -292,7 +292,7 @@ def run_ours(args, wl):
     pipe.submit(q_h, k_h, v_h, o_h, l_h)
     pipe.drain()
     barrier()
-    e2e_steps = max(1, min(args.steps, 20 if wl.seq_len <= 65536 else 4))
+    e2e_steps = max(1, min(args.steps, 20 if wl.seq_len <= 65536 else 8))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(pipe.s_in)                                       # nothing is in flight: first operation of the region
     for _ in range(e2e_steps):
