@@ -212,7 +212,8 @@ def run_ours(args, wl):
     if world == 1 and not args.no_extra and not args.profile:
         extra = {}
         for name, fn in (("c3", extra_partitioned), ("c3_merge_kernel", extra_merge_kernel), ("c4", run_preempted),
-                         ("c2", run_short_batch), ("ring", run_ring), ("decode", run_decode), ("linear", run_linear)):
+                         ("c2", run_short_batch), ("ring", run_ring), ("decode", run_decode), ("linear", run_linear),
+                         ("linear_merged", run_linear_merged)):
             try:
                 extra[name] = fn(args)
             except Exception as exc:                       # an extra record must not take the headline with it
@@ -561,6 +562,65 @@ def run_linear(args):
                       "max_abs_err_vs_oracle_sampled_rows": err}
 
 
+def run_linear_merged(args):
+    """Extra line: Eq. 5 on two unmerged partial results (the two GPUs' outputs of Section 5.2) in one call, beside
+    the same work as a merge pass followed by the plain GEMM."""
+    from paper_2409_15104_b200 import binding
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    M, hq, N, n = 32768, 32, 4096, 2
+    K = hq * 128
+    seed = workloads.BASE_SEED + 8
+    os_ = [workloads.normal_tensor(seed + i, 1, (M, hq, 128), torch.float32).to(dev) for i in range(n)]
+    ls_ = [(workloads.normal_tensor(seed + i, 2, (M, hq), torch.float32) * 2.0).to(dev) for i in range(n)]
+    w = (workloads.normal_tensor(seed, 3, (N, K), torch.float32) / K ** 0.5).to(torch.bfloat16).to(dev)
+    y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    o_m = torch.empty((M, hq, 128), dtype=torch.bfloat16, device=dev)
+    l_m = torch.empty((M, hq), dtype=torch.float32, device=dev)
+
+    def fused():
+        binding.pec_linear_merged(os_, ls_, w, y=y)
+
+    def two_calls():
+        binding.pec_attn_merge_n(os_, ls_, out_dtype=torch.bfloat16, o_out=o_m, lse_out=l_m)
+        binding.pec_linear(o_m.view(M, K), w, y=y)
+
+    steps = _extra_steps(args, 30)
+    ms = {}
+    for name, fn in (("two_calls", two_calls), ("fused", fused)):
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        binding.check_status()
+        ms[name] = e0.elapsed_time(e1) / steps
+    tf = 2.0 * M * N * K / (ms["fused"] * 1e-3) / 1e12
+    peaks = load_peaks()
+    import oracle
+    rows = [0, 1, 127, 128, 4095, M - 1]
+    merged, _ = oracle.merge_n([o[rows].cpu().numpy() for o in os_], [l[rows].cpu().numpy() for l in ls_])
+    want = oracle.linear(torch.from_numpy(merged.reshape(len(rows), K)), w.cpu())
+    err = float(np.abs(y[rows].float().cpu().double().numpy() - want).max())
+    col_tiles = (N + 511) // 512
+    l2_bytes = col_tiles * n * M * K * 4 + ((M + 255) // 256) * N * K * 2
+    return {"metric": "Eq. 5 on two unmerged partials, TFLOP/s of the GEMM (extra line, not the headline)", "value": tf,
+            "unit": "TFLOP/s", "ms_per_step": ms["fused"], "steps": steps, "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"linear_merged: {n} partials [{M},{hq},128] fp32 times w [{N},{K}]^T",
+                       "l2": "partials (1.07 GB) exceed L2"},
+            "ms_merge_pass_then_gemm": ms["two_calls"],
+            "operand_reads_through_l2": {"bytes": l2_bytes, "gbs": l2_bytes / (ms["fused"] * 1e-3) / 1e9,
+                                         "note": "every 512-column tile re-reads its rows of the fp32 partials"},
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+                         "frac": tf / peaks["bf16_sustained"], "traffic": None,
+                         "peak_source": peaks["source"] + " sustained cuBLAS bf16"},
+            "max_abs_err_vs_oracle_sampled_rows": err}
+
+
 def _short_batch(wl, dev, seed_offset=0):
     lens = workloads.short_lengths(wl.seed, wl.short_batch)
     cu = workloads.cu_seqlens(lens)
@@ -750,7 +810,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode", "linear", "ring", "merge"], default="c5",
+    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode", "linear", "linear_merged", "ring", "merge"], default="c5",
                     help="c5 (default, the largest single-GPU configuration) and c3 print the full line; the others "
                          "print their extra record alone")
     ap.add_argument("--no-extra", action="store_true", help="skip the extra records nested under the headline line")
@@ -765,7 +825,7 @@ def main():
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
-    alone = {"decode": run_decode, "linear": run_linear, "ring": run_ring, "c2": run_short_batch, "c4": run_preempted,
+    alone = {"decode": run_decode, "linear": run_linear, "linear_merged": run_linear_merged, "ring": run_ring, "c2": run_short_batch, "c4": run_preempted,
              "merge": extra_merge_kernel}
     if args.workload in alone:
         print(json.dumps(alone[args.workload](args)), flush=True)

@@ -388,6 +388,27 @@ int pec_linear(const void *x, int64_t x_stride, const void *w, int64_t w_stride,
                int64_t M, int32_t N, int32_t K, int32_t *status, void *cuda_stream);
 
 /*
+ * The post-self-attention linear layer (Eq. 5) taking partial attention results as they are:
+ *     y = merge(o_1 .. o_n) w^T,   merge as in pec_attn_merge_n:
+ *     lse = ln sum_i exp(lse_i);   o = sum_i exp(lse_i - lse) * o_i   per (row, head),
+ * the merged o rounded to bf16 (nearest even) as the GEMM's operand and never written to memory.
+ * This is what the GPU that finishes a shared long request does with its own and its peer's
+ * outputs O_1, O_2 in Section 5.2's colocation example (n = 2), or a GPU holding the partials of
+ * n key partitions (Section 2.2).
+ * o_parts / lse_parts: HOST arrays of n DEVICE pointers (1 <= n <= PEC_LINEAR_MERGED_MAX_PARTS),
+ * [rows, Hq, D] fp32 and [rows, Hq] fp32, contiguous, o 16-byte aligned; the arrays are read
+ * during the call only.  A part whose lse is -inf for a (row, head) is not read there; where
+ * every part's is, the merged row is 0.  D must be 128; the contraction runs over K = Hq * D.
+ * w: device [N, K] bf16, y: device [rows, N] bf16; row strides in elements (multiples of 8),
+ * 16-byte aligned; N a multiple of 8.  `status`: required device word, used as in pec_attn_args.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.
+ */
+#define PEC_LINEAR_MERGED_MAX_PARTS 8
+int pec_linear_merged(const void *const *o_parts, const float *const *lse_parts, int32_t n, int64_t rows, int32_t Hq,
+                      int32_t D, const void *w, int64_t w_stride, void *y, int64_t y_stride, int32_t N,
+                      int32_t *status, void *cuda_stream);
+
+/*
  * Process-wide settings (the paper has no counterpart; they exist for operations and tests).
  *   PEC_CTL_WAIT_LIMIT_CYCLES   limit of every barrier wait inside the kernels, in SM clock cycles
  *                               (default 2e9, about a second).  A wait that runs out makes its CTA
@@ -397,7 +418,7 @@ int pec_linear(const void *x, int64_t x_stride, const void *w, int64_t w_stride,
  *                               preemption works between kernels only) sets it lower.  value >= 1000.
  *   PEC_CTL_TEST_SKIP_LAST_LOAD test hook, 0 / 1: the loader of the tensor-core kernels leaves out its
  *                               last tile (attention: the last V tile of a CTA that walks at least two
- *                               key tiles; pec_linear: the last K step of the second CTA of each pair),
+ *                               key tiles; pec_linear, pec_linear_merged: the last K step of the second CTA of each pair),
  *                               so that the waits for it run out and the timeout path can be checked.
  *                               Results of such a launch are undefined; the status word tells.
  * Applies to launches enqueued after the call.  Errors: INVALID_ARG.

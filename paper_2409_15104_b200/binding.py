@@ -93,10 +93,12 @@ class pec_plan(ctypes.Structure):
 
 EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_attn_merge_n", "pec_plan_partitions",
            "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size", "pec_decode_attn_static", "pec_select_sp", "pec_linear",
-           "pec_plan_ring", "pec_balance_batches", "pec_plan_worklist", "pec_worklist_block_m", "pec_control")
+           "pec_plan_ring", "pec_balance_batches", "pec_plan_worklist", "pec_worklist_block_m", "pec_control",
+           "pec_linear_merged")
 PEC_CTL_WAIT_LIMIT_CYCLES, PEC_CTL_TEST_SKIP_LAST_LOAD = 1, 2
 PEC_DECODE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 PEC_MERGE_MAX_PARTS = 16
+PEC_LINEAR_MERGED_MAX_PARTS = 8
 
 
 def load():
@@ -132,6 +134,10 @@ def load():
     lib.pec_linear.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
                                ctypes.c_void_p]
+    lib.pec_linear_merged.restype = ctypes.c_int
+    lib.pec_linear_merged.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p), ctypes.c_int32,
+                                      ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int64,
+                                      ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
     lib.pec_select_sp.restype = ctypes.c_int
     lib.pec_select_sp.argtypes = [ctypes.POINTER(pec_sp_inputs), ctypes.POINTER(pec_sp_choice)]
     lib.pec_plan_ring.restype = ctypes.c_int
@@ -365,6 +371,26 @@ def pec_linear(x, w, y=None, stream=None):
     assert y.stride(1) == 1
     _check(lib.pec_linear(x.data_ptr(), x.stride(0), w.data_ptr(), w.stride(0), y.data_ptr(), y.stride(0), M, N, K,
                           status_word(x.device).data_ptr(), _stream_ptr(stream)))
+    return y
+
+
+def pec_linear_merged(o_parts, lse_parts, w, y=None, stream=None):
+    """y = merge(o_parts, lse_parts) w^T: fp32 partials [rows,Hq,128] with LSEs [rows,Hq], w [N,Hq*128] bf16; returns y [rows,N] bf16."""
+    lib = load()
+    n = len(o_parts)
+    assert n == len(lse_parts)
+    rows, Hq, D = o_parts[0].shape
+    for t in list(o_parts) + list(lse_parts):
+        assert t.is_cuda and t.is_contiguous() and t.dtype == torch.float32
+    assert w.is_cuda and w.dtype == torch.bfloat16 and w.stride(1) == 1 and w.shape[1] == Hq * D
+    N = w.shape[0]
+    if y is None:
+        y = torch.empty((rows, N), dtype=torch.bfloat16, device=w.device)
+    assert y.stride(1) == 1
+    op = (ctypes.c_void_p * n)(*[t.data_ptr() for t in o_parts])
+    lp = (ctypes.c_void_p * n)(*[t.data_ptr() for t in lse_parts])
+    _check(lib.pec_linear_merged(op, lp, n, rows, Hq, D, w.data_ptr(), w.stride(0), y.data_ptr(), y.stride(0), N,
+                                 status_word(w.device).data_ptr(), _stream_ptr(stream)))
     return y
 
 

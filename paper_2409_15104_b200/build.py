@@ -6,7 +6,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libpec.so")
-SOURCES = ["pec_api.cpp", "pec_plan.cpp", "pec_merge.cu", "pec_attn_f32.cu", "pec_attn_prefill_bf16.cu", "pec_attn_split_bf16.cu", "pec_decode.cu", "pec_linear.cu"]
+SOURCES = ["pec_api.cpp", "pec_plan.cpp", "pec_merge.cu", "pec_attn_f32.cu", "pec_attn_prefill_bf16.cu", "pec_attn_split_bf16.cu", "pec_decode.cu", "pec_linear.cu", "pec_linear_merged.cu"]
 
 
 def _stale() -> bool:

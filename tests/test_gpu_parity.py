@@ -343,6 +343,63 @@ def test_attention_layer_steps_chain_through_strides(pec):
     assert np.abs(out.float().cpu().double().numpy() - oracle.linear(o.view(T, hq * 128).cpu(), w_l)).max() <= 2e-2
 
 
+def _random_partials(seed, rows, hq, n):
+    """n fp32 partials with LSEs; about a fifth of the (row, head, part) entries empty (lse = -inf, o poisoned with NaN:
+    an empty part must not be read), and a few rows empty in every part."""
+    g = torch.Generator().manual_seed(seed)
+    os_, ls_ = [], []
+    dead_rows = torch.rand((rows, 1), generator=g) < 0.03
+    for i in range(n):
+        o = workloads.normal_tensor(seed + 10 * i, 1, (rows, hq, 128), torch.float32)
+        l = workloads.normal_tensor(seed + 10 * i + 1, 2, (rows, hq), torch.float32) * 3.0
+        empty = (torch.rand((rows, hq), generator=g) < 0.2) | dead_rows
+        l[empty] = float("-inf")
+        o[empty] = float("nan")
+        os_.append(o)
+        ls_.append(l)
+    return os_, ls_
+
+
+@pytest.mark.parametrize("rows,hq,N,n", [(1, 1, 8, 1), (100, 1, 72, 2), (256, 2, 512, 2), (300, 4, 520, 3), (700, 3, 1024, 4),
+                                         (513, 2, 1288, 8), (2048, 32, 4096, 2)])
+def test_linear_merged_matches_oracle(pec, rows, hq, N, n):
+    """Eq. 5 on the merge of n partials (Section 2.2, Section 5.2): against merge_n -> linear of the oracle."""
+    os_, ls_ = _random_partials(17000 + rows + n, rows, hq, n)
+    K = hq * 128
+    w = (workloads.normal_tensor(17001 + N, 3, (N, K), torch.float32) / K ** 0.5).to(torch.bfloat16)
+    merged, _ = oracle.merge_n([torch.nan_to_num(o, nan=0.0).numpy() for o in os_], [l.numpy() for l in ls_])
+    want = oracle.linear(torch.from_numpy(merged.reshape(rows, K)), w)
+    y = pec.pec_linear_merged([o.to(DEV) for o in os_], [l.to(DEV) for l in ls_], w.to(DEV))
+    pec.check_status()
+    got = y.float().cpu().double().numpy()
+    assert np.isfinite(got).all()
+    err = np.abs(got - want).max()
+    print(f"[parity] linear_merged rows={rows} Hq={hq} N={N} n={n}: max|dy| = {err:.3e}")
+    assert err <= 2e-2                                   # bf16 rounding of the merged operand and of the result
+    # the unfused route through the merge kernel and pec_linear rounds the same merged values the same way
+    if n >= 2:
+        o_m, _ = pec.pec_attn_merge_n([torch.nan_to_num(o, nan=0.0).to(DEV) for o in os_], [l.to(DEV) for l in ls_],
+                                      out_dtype=torch.bfloat16)
+        y2 = pec.pec_linear(o_m.view(rows, K), w.to(DEV))
+        pec.check_status()
+        assert (y2.float() - y.float()).abs().max().item() <= 2e-2
+
+
+def test_linear_merged_on_partitioned_attention(pec):
+    """Two key partitions' partial attention (the two GPUs' O_1, O_2 of Section 5.2) go into Eq. 5 unmerged."""
+    S, hq, hkv, d = 1536, 4, 2, 384
+    q, k, v = _qkv(workloads.BASE_SEED + 170, S, hq, hkv, torch.bfloat16)
+    w_l = (workloads.normal_tensor(17100, 3, (d, hq * 128), torch.float32) / (hq * 128) ** 0.5).to(torch.bfloat16)
+    parts = [pec.pec_prefill_attn(*_gpu(q, k, v), part_id=i, num_parts=2, part_align=64, out_dtype=torch.float32) for i in range(2)]
+    y = pec.pec_linear_merged([o for o, _ in parts], [l for _, l in parts], w_l.to(DEV))
+    pec.check_status()
+    want_o, _ = oracle.prefill_attn(q, k, v, seq_len=S)
+    want = oracle.linear(torch.from_numpy(np.asarray(want_o).reshape(S, hq * 128)), w_l)
+    err = np.abs(y.float().cpu().double().numpy() - want).max()
+    print(f"[parity] attention partials -> linear_merged: max|dy| = {err:.3e}")
+    assert err <= 2e-2
+
+
 # ------------------------------------------------------------------ ring-attention step form
 @pytest.mark.parametrize("S,P,hq,hkv", [(2048, 4, 4, 2), (1500, 3, 2, 1), (700, 1, 2, 2), (300, 8, 2, 1)])
 def test_ring_prefill_every_rank_and_step_equals_monolithic(pec, S, P, hq, hkv):

@@ -60,6 +60,26 @@ def test_linear_pair_leaves_together_when_a_wait_runs_out(pec, short_waits):
     assert np.abs(y.float().cpu().double().numpy() - oracle.linear(x, w)).max() <= 2e-2
 
 
+def test_linear_merged_pair_leaves_together_when_a_wait_runs_out(pec, short_waits):
+    rows, hq, N = 256, 1, 512                                 # one CTA pair, two K steps
+    os_ = [workloads.normal_tensor(21010 + i, 1, (rows, hq, 128), torch.float32) for i in range(2)]
+    ls_ = [workloads.normal_tensor(21020 + i, 2, (rows, hq), torch.float32) for i in range(2)]
+    w = (workloads.normal_tensor(21003, 3, (N, hq * 128), torch.float32) / 128 ** 0.5).to(torch.bfloat16)
+    do, dl, dw = [o.to(DEV) for o in os_], [l.to(DEV) for l in ls_], w.to(DEV)
+    pec.check_status()
+    pec.pec_linear_merged(do, dl, dw)                         # the second CTA's last K step of w never arrives
+    torch.cuda.synchronize()
+    with pytest.raises(pec.PecError) as err:
+        pec.check_status()
+    assert err.value.code == pec.PEC_ERR_TIMEOUT
+    pec.pec_control(pec.PEC_CTL_TEST_SKIP_LAST_LOAD, 0)
+    y = pec.pec_linear_merged(do, dl, dw)
+    pec.check_status()
+    merged, _ = oracle.merge_n([o.numpy() for o in os_], [l.numpy() for l in ls_])
+    want = oracle.linear(torch.from_numpy(merged.reshape(rows, hq * 128)), w)
+    assert np.abs(y.float().cpu().double().numpy() - want).max() <= 2e-2
+
+
 def test_control_rejects_unknown_settings(pec):
     with pytest.raises(pec.PecError):
         pec.pec_control(99, 1)

@@ -167,6 +167,23 @@ def test_decode_validates_on_the_host_and_sizes_its_workspace():
         setattr(a, field, old)
 
 
+def test_linear_merged_validates_on_the_host():
+    import ctypes
+    f = binding.load().pec_linear_merged
+
+    def call(o=(4096, 8192), l=(256, 512), n=2, rows=10, Hq=1, D=128, w=16384, ws=128, y=32768, ys=32, N=32, st=65536):
+        op = (ctypes.c_void_p * max(len(o), 1))(*o)
+        lp = (ctypes.c_void_p * max(len(l), 1))(*l)
+        return f(op, lp, n, rows, Hq, D, w, ws, y, ys, N, st, None)
+
+    assert call(rows=0) == 0
+    assert call(n=0) == -1 and call(n=9, o=(4096,) * 9, l=(256,) * 9) == -1 and call(st=None) == -1 and call(w=None) == -1
+    assert call(o=(4096, None)) == -1 and call(rows=-1) == -1 and call(Hq=0) == -1 and call(N=0) == -1
+    assert call(D=64) == -2 and call(N=36) == -2
+    assert call(ws=64) == -1 and call(ys=16) == -1
+    assert call(o=(4100, 8192)) == -3 and call(ws=132) == -3 and call(y=32772) == -3
+
+
 def test_linear_validates_on_the_host():
     f = binding.load().pec_linear
     ok = dict(x=4096, xs=64, w=8192, ws=64, y=12288, ys=32, M=10, N=32, K=64, st=16384)
