@@ -75,40 +75,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     return true;
 }
 
-// Cluster-scope forms for a barrier that threads of the partner CTA arrive on after writing their own
-// shared memory with ordinary stores: the arrive releases, the wait acquires, both at cluster scope.
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_suspend_cluster(uint32_t bar, uint32_t parity, uint32_t ns)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_bounded_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag, int32_t *status,
-                                                          long long limit_cycles, int timeout_code)
-{
-    const long long t0 = clock64();
-    while (!mbar_try_wait_suspend_cluster(bar, parity, 2000u)) {
-        if (*abort_flag) return false;
-        if (clock64() - t0 > limit_cycles) {
-            *abort_flag = 1;
-            if (status) atomicExch(status, timeout_code);
-            return false;
-        }
-    }
-    return true;
-}
-// Orders this thread's ordinary shared-memory stores before later reads of the same memory by the async
-// proxy (TMA, tcgen05.mma operands).
-__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
 // ---------------------------------------------------------------- programmatic dependent launch
 // launch_dependents: once every CTA of this grid has executed it (or exited), a following kernel that was launched
 // as a programmatic dependent may start on SMs this grid no longer needs.  wait: blocks until the kernel(s) this grid
