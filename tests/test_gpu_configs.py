@@ -179,3 +179,31 @@ def test_c3_every_row_against_the_fp32_kernel(pec):
     wl = workloads.WORKLOADS["c3"]
     q, k, v, o, lse = _merged_result(pec, "c3")
     _cross_check_all_rows(pec, o, lse, q, k, v, list(range(wl.hq)), "c3")
+
+
+# ------------------------------------------------------------------ the paper's longest inputs
+def test_longest_paper_input_500k_ragged_eight_partitions_and_last_chunk(pec):
+    """Section 6.1 draws long inputs from up to 500K tokens.  S = 500,000 is not a multiple of the tile (the last
+    key tile holds 32 keys), of the chunk or of 2 * P * align; one KV head serves eight query heads.  The
+    partitioned path over eight zigzag partitions and, separately, the last preemptible chunk resumed from
+    the whole stored prefix are compared with the oracle on sampled rows."""
+    S, hq, hkv, P, C = 500_000, 8, 1, 8, 8192
+    q, k, v = workloads.qkv(workloads.BASE_SEED + 500, S, hq, hkv, 128, torch.bfloat16)
+    dq, dk, dv = q.to(DEV), k.to(DEV), v.to(DEV)
+    plan = pec.pec_plan_partitions(S, P, C, 128, 128, 128, True, tiles=False)
+    want_plan = oracle.plan_partitions(S, P, C, 128, 128, 128, True, tiles=False)
+    assert plan["bounds"] == want_plan["bounds"] and plan["pairs"] == want_plan["pairs"] and plan["chunks"] == want_plan["chunks"]
+    assert sum(plan["pairs"]) == S * (S + 1) // 2
+    runner = PartitionedPrefill(S, hq, P, torch.bfloat16, DEV, 128)
+    o, lse = runner.run(dq, dk, dv)
+    pec.check_status()
+    tail = (S // 128) * 128
+    rows = sample_rows(S, list(plan["bounds"][::2]) + [tail, S - 2], 40, 500)
+    _check_sampled(o, lse, q, k, v, S, rows, torch.bfloat16, "S=500000 merged")
+    c0 = (S // C) * C                                          # last chunk: 288 rows
+    oc, lc = pec.pec_prefill_attn(dq, dk, dv, seq_len=S, chunk_start=c0, chunk_len=S - c0, kv_len=S)
+    pec.check_status()
+    crow = sample_rows(S, [tail], 8, 501, lo=c0, hi=S)
+    want = oracle.prefill_attn(q, k, v, seq_len=S, rows=crow)
+    idx = torch.as_tensor([r - c0 for r in crow], device=DEV)
+    compare(oc[idx], lc[idx], *want, *TOL[torch.bfloat16], "S=500000 last chunk")
