@@ -12,6 +12,8 @@ from .reference import (  # noqa: F401
     sp_volumes,
     select_sp,
     linear,
+    rope,
+    linear_rope,
     plan_partitions,
     plan_worklist,
     partition_rows,

@@ -377,3 +377,33 @@ def linear(x, w):
     """y = x w^T in fp64 (numpy matmul): QKV generation (Eq. 2) with the per-head weights stacked
     row-wise in w, or the post-self-attention linear layer (Eq. 5) with w = W_L^T."""
     return _as_f32(x).astype(np.float64) @ _as_f32(w).astype(np.float64).T
+
+
+def rope(y, positions, theta, rot_cols, head_dim=128):
+    """Rotary position encoding of the leading rot_cols columns of y [T, N] (fp64 numpy).  The paper
+    never states a position encoding; the Llama models it serves (Section 6.1) use the rotary form of
+    RoFormer in its "rotate-half" pairing, which is what this restates: the columns are heads of
+    head_dim channels, channel i < head_dim/2 of a head pairs with channel i + head_dim/2, and the
+    pair of the token at position p is turned by the angle p * theta**(-2 i / head_dim):
+        out[i]       = y[i] cos - y[i + d/2] sin
+        out[i + d/2] = y[i + d/2] cos + y[i] sin.
+    Columns from rot_cols on (the values) are returned unchanged."""
+    out = _as_f32(y).astype(np.float64) if hasattr(y, "detach") else np.array(y, dtype=np.float64, copy=True)
+    pos = np.asarray(positions, dtype=np.float64).reshape(-1)
+    assert out.shape[0] == pos.shape[0] and rot_cols % head_dim == 0 and rot_cols <= out.shape[1]
+    half = head_dim // 2
+    inv_freq = np.float64(theta) ** (-2.0 * np.arange(half, dtype=np.float64) / head_dim)
+    ang = pos[:, None] * inv_freq[None, :]                                     # [T, d/2]
+    c, s_ = np.cos(ang), np.sin(ang)
+    for h0 in range(0, rot_cols, head_dim):
+        a = out[:, h0:h0 + half].copy()
+        b = out[:, h0 + half:h0 + head_dim].copy()
+        out[:, h0:h0 + half] = a * c - b * s_
+        out[:, h0 + half:h0 + head_dim] = b * c + a * s_
+    return out
+
+
+def linear_rope(x, w, positions, theta, rot_cols, head_dim=128):
+    """QKV generation (Eq. 2) followed by the rotary encoding of the query and key heads."""
+    return rope(linear(x, w), positions, theta, rot_cols, head_dim)
+

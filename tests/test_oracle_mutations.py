@@ -131,6 +131,13 @@ PY_MUTATIONS = {
     "work-list ties by position before request": ("entries.sort(key=lambda e: e[:3])", "entries.sort(key=lambda e: (e[0], e[2], e[1]))"),
     "work-list last tile not cut": ("n = min(block_m, L - pos0)", "n = block_m"),
     "partition rows ignore the chunk start": ("range(max(lo, chunk_start), min(hi, chunk_start + chunk_len))", "range(lo, min(hi, chunk_start + chunk_len))"),
+    "rope turns the other way": ("out[:, h0:h0 + half] = a * c - b * s_", "out[:, h0:h0 + half] = a * c + b * s_"),
+    "rope second half without the cross term": ("out[:, h0 + half:h0 + head_dim] = b * c + a * s_", "out[:, h0 + half:h0 + head_dim] = b * c"),
+    "rope frequency exponent i/d": ("** (-2.0 * np.arange(half, dtype=np.float64) / head_dim)", "** (-1.0 * np.arange(half, dtype=np.float64) / head_dim)"),
+    "rope pairs neighbouring channels": ("        a = out[:, h0:h0 + half].copy()\n        b = out[:, h0 + half:h0 + head_dim].copy()\n        out[:, h0:h0 + half] = a * c - b * s_\n        out[:, h0 + half:h0 + head_dim] = b * c + a * s_",
+                                         "        a = out[:, h0:h0 + head_dim:2].copy()\n        b = out[:, h0 + 1:h0 + head_dim:2].copy()\n        out[:, h0:h0 + head_dim:2] = a * c - b * s_\n        out[:, h0 + 1:h0 + head_dim:2] = b * c + a * s_"),
+    "rope turns the values too": ("for h0 in range(0, rot_cols, head_dim):", "for h0 in range(0, out.shape[1], head_dim):"),
+    "rope angle from the row index": ("ang = pos[:, None] * inv_freq[None, :]", "ang = np.arange(len(pos), dtype=np.float64)[:, None] * inv_freq[None, :]"),
     "MLP parameter volume 4 d^2": ("(8 * d * d * (T - 1) * G / T, 16 * s * d * d)", "(4 * d * d * (T - 1) * G / T, 16 * s * d * d)"),
 }
 
@@ -146,7 +153,7 @@ def test_a_mistake_in_the_python_oracle_is_caught(name, monkeypatch):
     exec(compile(src.replace(old, new), "reference_mutant.py", "exec"), mod.__dict__)
     for attr in ("attn_rows", "prefill_attn", "varlen_attn", "merge", "merge_n", "plan_partitions",
                  "partition_intervals", "sp_volumes", "select_sp", "linear", "plan_ring", "ring_segments",
-                 "balance_batches", "plan_worklist", "partition_rows"):
+                 "balance_batches", "plan_worklist", "partition_rows", "rope", "linear_rope"):
         monkeypatch.setattr(oracle, attr, getattr(mod, attr))
     # The ring/batch pin file also compares the library with the oracle; here the library is replaced by an
     # echo of the mutant, so that only the pins proper (enumeration, hand-worked values, bounds) can object.

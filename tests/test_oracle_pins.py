@@ -349,3 +349,65 @@ def test_linear_matches_loops_identity_and_per_head_stacking():
     both = oracle.linear(x, np.concatenate([wq, wk]))
     np.testing.assert_array_equal(both[:, :3], oracle.linear(x, wq))
     np.testing.assert_array_equal(both[:, 3:], oracle.linear(x, wk))
+
+
+# --------------------------------------------------------------------------- rotary position encoding
+def test_rope_matches_the_hand_worked_rotations():
+    path = os.path.join(os.path.dirname(__file__), "golden", "rope_worked.txt")
+    n = 0
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        head, vec, want = (part.split() for part in line.split("|"))
+        d, theta, pos = int(head[0]), float(head[1]), int(head[2])
+        got = oracle.rope(np.array([[float(x) for x in vec]]), [pos], theta, d, head_dim=d)
+        np.testing.assert_allclose(got[0], [float(x) for x in want], rtol=0, atol=1e-14)
+        n += 1
+    assert n == 3
+
+
+def test_rope_is_a_rotation_that_depends_on_relative_position_only():
+    g = np.random.Generator(np.random.Philox(key=77))
+    d, theta = 128, 500000.0
+    qv, kv = g.standard_normal((1, 2 * d)), g.standard_normal((1, 2 * d))
+    # position 0 changes nothing
+    np.testing.assert_array_equal(oracle.rope(qv, [0], theta, 2 * d, d), qv)
+    # every (i, i + d/2) pair keeps its length
+    r = oracle.rope(qv, [12345], theta, 2 * d, d)
+    for h0 in (0, d):
+        before = qv[0, h0:h0 + d // 2] ** 2 + qv[0, h0 + d // 2:h0 + d] ** 2
+        after = r[0, h0:h0 + d // 2] ** 2 + r[0, h0 + d // 2:h0 + d] ** 2
+        np.testing.assert_allclose(after, before, rtol=1e-12)
+    # q.k after the encoding depends on the distance of the two positions only (per head)
+    for m, n in ((700, 300), (40000, 39600), (5, 405)):
+        a = oracle.rope(qv, [m], theta, 2 * d, d)[0, :d] @ oracle.rope(kv, [n], theta, 2 * d, d)[0, :d]
+        b = oracle.rope(qv, [m - n + 1000], theta, 2 * d, d)[0, :d] @ oracle.rope(kv, [1000], theta, 2 * d, d)[0, :d]
+        np.testing.assert_allclose(a, b, rtol=0, atol=1e-9)
+    # turning by a and then by b is turning by a + b
+    twice = oracle.rope(oracle.rope(qv, [17], theta, 2 * d, d), [25], theta, 2 * d, d)
+    np.testing.assert_allclose(twice, oracle.rope(qv, [42], theta, 2 * d, d), rtol=0, atol=1e-12)
+    # the slowest pair of a head turns by position / theta**((d-2)/d): a quarter turn there swaps the pair
+    pos = (np.pi / 2) * theta ** ((d - 2) / d)
+    e = np.zeros((1, d)); e[0, d // 2 - 1] = 1.0
+    out = oracle.rope(e, [pos], theta, d, d)
+    np.testing.assert_allclose([out[0, d // 2 - 1], out[0, d - 1]], [0.0, 1.0], rtol=0, atol=1e-9)
+
+
+def test_rope_leaves_the_value_columns_alone_and_shares_angles_between_heads():
+    g = np.random.Generator(np.random.Philox(key=78))
+    d = 128
+    y = g.standard_normal((5, 4 * d))
+    pos = [0, 1, 2, 1000, 77]
+    out = oracle.rope(y, pos, 10000.0, 3 * d, d)
+    np.testing.assert_array_equal(out[:, 3 * d:], y[:, 3 * d:])
+    assert not np.allclose(out[1:, :3 * d], y[1:, :3 * d])
+    # the same vector in two heads comes out the same
+    y2 = np.concatenate([y[:, :d], y[:, :d]], axis=1)
+    o2 = oracle.rope(y2, pos, 10000.0, 2 * d, d)
+    np.testing.assert_array_equal(o2[:, :d], o2[:, d:])
+    # rows are independent: a row's result depends on its own position only
+    np.testing.assert_array_equal(oracle.rope(y[3:4], [1000], 10000.0, 3 * d, d), out[3:4])
+    # linear_rope is the encoding of the projection
+    x, w = g.standard_normal((5, 16)).astype(np.float32), g.standard_normal((4 * d, 16)).astype(np.float32)
+    np.testing.assert_array_equal(oracle.linear_rope(x, w, pos, 10000.0, 3 * d, d), oracle.rope(oracle.linear(x, w), pos, 10000.0, 3 * d, d))
+
