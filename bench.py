@@ -553,7 +553,24 @@ def run_linear(args):
     rows = [0, 1, 127, 128, 4095, M - 1]
     want = oracle.linear(x[rows].cpu(), w.cpu())
     err = float(np.abs(y[rows].float().cpu().double().numpy() - want).max())
+    # The same GEMM with the rotary position encoding of the query and key heads in its epilogue.
+    theta, rot_cols = 500000.0, (32 + 8) * 128
+    tables = binding.pec_rope_table(theta, M, dev)
+    for _ in range(3):
+        binding.pec_linear_rope(x, w, tables, rot_cols, y=y)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        binding.pec_linear_rope(x, w, tables, rot_cols, y=y)
+    e1.record()
+    torch.cuda.synchronize()
+    binding.check_status()
+    ms_rope = e0.elapsed_time(e1) / steps
+    want = oracle.linear_rope(x[rows].cpu(), w.cpu(), rows, theta, rot_cols)
+    err_rope = float(np.abs(y[rows].float().cpu().double().numpy() - want).max())
     return {"metric": "QKV-generation GEMM TFLOP/s (extra line, not the headline)", "value": tf, "unit": "TFLOP/s",
+            "with_rotary_encoding": {"ms_per_step": ms_rope, "tflops": 2.0 * M * N * K / (ms_rope * 1e-3) / 1e12,
+                                     "max_abs_err_vs_oracle_sampled_rows": err_rope},
                       "ms_per_step": ms, "steps": steps, "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
                       "config": {"workload": f"linear: x [{M},{K}] times w [{N},{K}]^T", "l2": "operands and output (752 MB) exceed L2"},
                       "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",

@@ -388,6 +388,34 @@ int pec_linear(const void *x, int64_t x_stride, const void *w, int64_t w_stride,
                int64_t M, int32_t N, int32_t K, int32_t *status, void *cuda_stream);
 
 /*
+ * QKV generation (Eq. 2) with rotary position encoding of the query and key heads applied to the
+ * fp32 accumulator before it is rounded to bf16.  The paper states no position encoding; the Llama
+ * models it serves (Section 6.1) use this one (RoFormer's rotation in its "rotate-half" pairing):
+ * the leading rot_cols columns of y are heads of 128 channels, channel i < 64 of a head pairs with
+ * channel i + 64, and for the row at position p
+ *     y'[i]      = y[i] cos(a) - y[i + 64] sin(a)
+ *     y'[i + 64] = y[i + 64] cos(a) + y[i] sin(a),      a = p * theta^(-2 i / 128).
+ * Columns from rot_cols on (the value heads) are left as they are.  rot_cols: multiple of 128, <= N.
+ * rope_cos / rope_sin: device [n_pos, 64] fp32 tables of cos(a) and sin(a) (pec_rope_table fills
+ * them), 16-byte aligned.  Row r is at position positions[r] (device int32 [M], e.g. a packed
+ * batch's positions within their requests) or, with positions == NULL, at pos0 + r (a chunk of one
+ * request, Section 5.1); positions outside [0, n_pos) are clamped to the table's ends, and the
+ * host rejects pos0 + M > n_pos.  Everything else as in pec_linear.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.
+ */
+int pec_linear_rope(const void *x, int64_t x_stride, const void *w, int64_t w_stride, void *y, int64_t y_stride,
+                    int64_t M, int32_t N, int32_t K, const float *rope_cos, const float *rope_sin, int64_t n_pos,
+                    const int32_t *positions, int64_t pos0, int32_t rot_cols, int32_t *status, void *cuda_stream);
+
+/*
+ * Fills the tables pec_linear_rope reads: cos_out[p][i] = cos(p * theta^(-2 i / D)),
+ * sin_out[p][i] likewise, for 0 <= p < n_pos, 0 <= i < D / 2, worked out in fp64 on the device
+ * and stored as fp32 (device [n_pos, D / 2] each).  D must be 128; theta > 0 (500000 for Llama-3).
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+int pec_rope_table(double theta, int64_t n_pos, int32_t D, float *cos_out, float *sin_out, void *cuda_stream);
+
+/*
  * The post-self-attention linear layer (Eq. 5) taking partial attention results as they are:
  *     y = merge(o_1 .. o_n) w^T,   merge as in pec_attn_merge_n:
  *     lse = ln sum_i exp(lse_i);   o = sum_i exp(lse_i - lse) * o_i   per (row, head),

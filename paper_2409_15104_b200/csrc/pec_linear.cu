@@ -45,10 +45,74 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Wa
     return mbar_wait_bounded(bar, parity, w.abort_flag, w.status, w.limit, (int)PEC_ERR_TIMEOUT);
 }
 
+// Rotary position encoding applied to the accumulator before it is rounded (kRope): the leading rot_cols
+// columns of y are heads of 128 channels; channel i < 64 of a head pairs with channel i + 64 and the pair of
+// the row at position p is turned by the angle whose cosine and sine are cos_tab[p][i], sin_tab[p][i].
+struct Rope {
+    const float *cos_tab, *sin_tab;                           // [n_pos, 64] fp32
+    const int32_t *positions;                                 // [M] or NULL: row r is at position pos0 + r
+    int64_t pos0;
+    int32_t n_pos, rot_cols;
+};
+
+// 32 accumulator columns -> bf16, 16 bytes per store, columns at or past N left out.
+__device__ __forceinline__ void store_chunk(__nv_bfloat16 *dst, const uint32_t (&r)[32], int col0, int32_t N)
+{
+#pragma unroll
+    for (int i = 0; i < 32; i += 8) {
+        if (col0 + i < N) {
+            uint4 pk;
+            pk.x = pack_bf16(__uint_as_float(r[i + 0]), __uint_as_float(r[i + 1]));
+            pk.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+            pk.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+            pk.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+            *reinterpret_cast<uint4 *>(dst + i) = pk;
+        }
+    }
+}
+
+__device__ __forceinline__ void store_chunk16(__nv_bfloat16 *dst, const uint32_t (&r)[16], int col0, int32_t N)
+{
+#pragma unroll
+    for (int i = 0; i < 16; i += 8) {
+        if (col0 + i < N) {
+            uint4 pk;
+            pk.x = pack_bf16(__uint_as_float(r[i + 0]), __uint_as_float(r[i + 1]));
+            pk.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+            pk.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+            pk.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+            *reinterpret_cast<uint4 *>(dst + i) = pk;
+        }
+    }
+}
+// Sixteen cosines and sines of a row, channels i0 .. i0 + 15 (row[0] = its line of the cosine table, row[1] of the sines).
+__device__ __forceinline__ void rope_fetch(const float *const (&row)[2], int i0, float4 (&c)[4], float4 (&s)[4])
+{
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+        c[v] = __ldg(reinterpret_cast<const float4 *>(row[0] + i0) + v);
+        s[v] = __ldg(reinterpret_cast<const float4 *>(row[1] + i0) + v);
+    }
+}
+// Two 16-column accumulator loads in flight, then one wait.
+__device__ __forceinline__ void tmem_ld16x2(uint32_t ta, uint32_t (&a)[16], uint32_t tb, uint32_t (&b)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%32];\n\t"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%33];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]), "=r"(a[4]), "=r"(a[5]), "=r"(a[6]), "=r"(a[7]),
+          "=r"(a[8]), "=r"(a[9]), "=r"(a[10]), "=r"(a[11]), "=r"(a[12]), "=r"(a[13]), "=r"(a[14]), "=r"(a[15]),
+          "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3]), "=r"(b[4]), "=r"(b[5]), "=r"(b[6]), "=r"(b[7]),
+          "=r"(b[8]), "=r"(b[9]), "=r"(b[10]), "=r"(b[11]), "=r"(b[12]), "=r"(b[13]), "=r"(b[14]), "=r"(b[15])
+        : "r"(ta), "r"(tb) : "memory");
+}
+
+template <bool kRope>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 2)
 linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t band, int32_t by_cols, int32_t *status,
-              long long wait_cycles, int32_t test_skip_last_load)
+              long long wait_cycles, int32_t test_skip_last_load, const Rope rope)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -137,26 +201,56 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
         }
         __syncwarp();
     } else {
+        const int64_t row = m0 + warp * 32 + lane;
+        [[maybe_unused]] const float *rope_row[2] = {nullptr, nullptr};
+        [[maybe_unused]] float4 c_next[4], s_next[4];
+        if constexpr (kRope) {
+            int64_t pos = 0;
+            if (row < M) pos = rope.positions ? (int64_t)rope.positions[row] : rope.pos0 + row;
+            pos = pos < 0 ? 0 : (pos >= rope.n_pos ? rope.n_pos - 1 : pos);
+            rope_row[0] = rope.cos_tab + pos * 64;
+            rope_row[1] = rope.sin_tab + pos * 64;
+            if (n0 < rope.rot_cols) rope_fetch(rope_row, 0, c_next, s_next);     // a tile of value heads needs none
+        }
         const bool ok = __all_sync(0xffffffffu, n_kb == 0 || wait_bar(smem_u32(&sh->acc_full), 0, wctx));
         if (ok) {
             tc_fence_after();
-            const int64_t row = m0 + warp * 32 + lane;
             const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+            if constexpr (!kRope) {
 #pragma unroll 1
-            for (int c = 0; c < kBN / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(taddr + c * 32, r);                 // warp-wide; only the stores are predicated
-                if (row < M) {
-                    __nv_bfloat16 *dst = y + row * y_stride + n0 + c * 32;
+                for (int c = 0; c < kBN / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(taddr + c * 32, r);             // warp-wide; only the stores are predicated
+                    if (row < M) store_chunk(y + row * y_stride + n0 + c * 32, r, n0 + c * 32, N);
+                }
+            } else {
+                // The tile's 256 columns are two heads; a thread holds a whole row, so both channels of a pair are its own.
+                // Sixteen pairs of both heads per step, so a row's cosines and sines are fetched once per tile; those of a
+                // step are asked for one step ahead (those of the first step before the wait for the accumulator).
+                const bool turn0 = n0 < rope.rot_cols, turn1 = n0 + 128 < rope.rot_cols;    // rot_cols: whole heads
+#pragma unroll 1
+                for (int it = 0; it < 4; ++it) {              // channels 16 it .. 16 it + 15 and their partners, both heads
+                    float4 c4[4], s4[4];
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        if (n0 + c * 32 + i < N) {
-                            uint4 pk;
-                            pk.x = pack_bf16(__uint_as_float(r[i + 0]), __uint_as_float(r[i + 1]));
-                            pk.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-                            pk.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-                            pk.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
-                            *reinterpret_cast<uint4 *>(dst + i) = pk;
+                    for (int v = 0; v < 4; ++v) { c4[v] = c_next[v]; s4[v] = s_next[v]; }
+                    if (it < 3 && turn0) rope_fetch(rope_row, (it + 1) * 16, c_next, s_next);
+                    const float *cf = reinterpret_cast<const float *>(c4), *sf = reinterpret_cast<const float *>(s4);
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
+                        const int col_a = hh * 128 + it * 16, col_b = col_a + 64;
+                        uint32_t a[16], b[16];
+                        tmem_ld16x2(taddr + col_a, a, taddr + col_b, b);
+                        if (hh == 0 ? turn0 : turn1) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float xa = __uint_as_float(a[j]), xb = __uint_as_float(b[j]);
+                                a[j] = __float_as_uint(xa * cf[j] - xb * sf[j]);
+                                b[j] = __float_as_uint(xb * cf[j] + xa * sf[j]);
+                            }
+                        }
+                        if (row < M) {
+                            store_chunk16(y + row * y_stride + n0 + col_a, a, n0 + col_a, N);
+                            store_chunk16(y + row * y_stride + n0 + col_b, b, n0 + col_b, N);
                         }
                     }
                 }
@@ -172,35 +266,67 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
 }  // namespace lin
 }  // namespace pec
 
+// cos and sin of position * theta^(-2 i / 128), i < 64, worked out in fp64 and stored as fp32.
+namespace pec {
+namespace lin {
+__global__ void rope_table_kernel(double log2_theta, int64_t n_pos, float *cos_out, float *sin_out)
+{
+    const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n_pos * 64) return;
+    const int i = (int)(idx & 63);
+    const double inv_freq = exp2(-(double)(2 * i) / 128.0 * log2_theta);
+    double s, c;
+    sincos((double)(idx >> 6) * inv_freq, &s, &c);
+    cos_out[idx] = (float)c;
+    sin_out[idx] = (float)s;
+}
+}  // namespace lin
+}  // namespace pec
+
 using namespace pec;
 
-extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_t w_stride, void *y, int64_t y_stride,
-                          int64_t M, int32_t N, int32_t K, int32_t *status, void *cuda_stream)
+static int linear_common(const char *who, const void *x, int64_t x_stride, const void *w, int64_t w_stride, void *y, int64_t y_stride,
+                         int64_t M, int32_t N, int32_t K, int32_t *status, void *cuda_stream, const lin::Rope *rope)
 {
-    if (!x || !w || !y || !status) { set_error("pec_linear: x, w, y and status must be non-NULL"); return PEC_ERR_INVALID_ARG; }
-    if (M < 0 || N < 1 || K < 1 || M >= ((int64_t)1 << 31)) { set_error("pec_linear: need 0 <= M < 2^31, N >= 1, K >= 1"); return PEC_ERR_INVALID_ARG; }
-    if (N % 8 != 0 || K % 8 != 0) { set_error("pec_linear: N and K must be multiples of 8"); return PEC_ERR_UNSUPPORTED; }
-    if (x_stride < K || w_stride < K || y_stride < N) { set_error("pec_linear: a row stride is smaller than the row"); return PEC_ERR_INVALID_ARG; }
+    if (!x || !w || !y || !status) { set_error("%s: x, w, y and status must be non-NULL", who); return PEC_ERR_INVALID_ARG; }
+    if (M < 0 || N < 1 || K < 1 || M >= ((int64_t)1 << 31)) { set_error("%s: need 0 <= M < 2^31, N >= 1, K >= 1", who); return PEC_ERR_INVALID_ARG; }
+    if (N % 8 != 0 || K % 8 != 0) { set_error("%s: N and K must be multiples of 8", who); return PEC_ERR_UNSUPPORTED; }
+    if (x_stride < K || w_stride < K || y_stride < N) { set_error("%s: a row stride is smaller than the row", who); return PEC_ERR_INVALID_ARG; }
     if (x_stride % 8 != 0 || w_stride % 8 != 0 || y_stride % 8 != 0 || (reinterpret_cast<uintptr_t>(x) & 15u) ||
         (reinterpret_cast<uintptr_t>(w) & 15u) || (reinterpret_cast<uintptr_t>(y) & 15u) || (reinterpret_cast<uintptr_t>(status) & 3u)) {
-        set_error("pec_linear: x, w, y must be 16-byte aligned with row strides that are multiples of 8 elements");
+        set_error("%s: x, w, y must be 16-byte aligned with row strides that are multiples of 8 elements", who);
         return PEC_ERR_ALIGNMENT;
+    }
+    if (rope) {
+        if (!rope->cos_tab || !rope->sin_tab || rope->n_pos < 1) { set_error("%s: the cos / sin tables must be non-NULL with n_pos >= 1", who); return PEC_ERR_INVALID_ARG; }
+        if (rope->rot_cols < 0 || rope->rot_cols > N) { set_error("%s: rot_cols must lie in [0, N]", who); return PEC_ERR_INVALID_ARG; }
+        if (rope->rot_cols % 128 != 0) { set_error("%s: rot_cols must be a multiple of 128 (whole heads)", who); return PEC_ERR_UNSUPPORTED; }
+        if (!rope->positions && (rope->pos0 < 0 || rope->pos0 + M > rope->n_pos)) {
+            set_error("%s: positions pos0 .. pos0 + M - 1 must lie inside the tables", who);
+            return PEC_ERR_INVALID_ARG;
+        }
+        if ((reinterpret_cast<uintptr_t>(rope->cos_tab) & 15u) || (reinterpret_cast<uintptr_t>(rope->sin_tab) & 15u) ||
+            (reinterpret_cast<uintptr_t>(rope->positions) & 3u)) {
+            set_error("%s: the cos / sin tables must be 16-byte aligned", who);
+            return PEC_ERR_ALIGNMENT;
+        }
     }
     if (M == 0) return PEC_OK;
     CUtensorMap tm_x, tm_w;
     if (!host::make_matrix_map(&tm_x, x, M, K, x_stride, lin::kBM) || !host::make_matrix_map(&tm_w, w, N, K, w_stride, 128)) {
-        set_error("pec_linear: cuTensorMapEncodeTiled failed");
+        set_error("%s: cuTensorMapEncodeTiled failed", who);
         return PEC_ERR_CUDA;
     }
     static unsigned char ready[host::kMaxDevices] = {};
     static std::mutex ready_mutex;
     if (!host::once_per_device(ready, ready_mutex, [] {
-            return cudaFuncSetAttribute(lin::linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::kSmemBytes) == cudaSuccess; })) {
-        set_error("pec_linear: cannot raise the shared-memory limit: %s", cudaGetErrorString(cudaGetLastError()));
+            return cudaFuncSetAttribute(lin::linear_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::kSmemBytes) == cudaSuccess &&
+                   cudaFuncSetAttribute(lin::linear_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::kSmemBytes) == cudaSuccess; })) {
+        set_error("%s: cannot raise the shared-memory limit: %s", who, cudaGetErrorString(cudaGetLastError()));
         return PEC_ERR_CUDA;
     }
     const int64_t pairs = (M + 2 * lin::kBM - 1) / (2 * lin::kBM), gn = (N + lin::kBN - 1) / lin::kBN;
-    if (gn > 65535) { set_error("pec_linear: N too large"); return PEC_ERR_UNSUPPORTED; }
+    if (gn > 65535) { set_error("%s: N too large", who); return PEC_ERR_UNSUPPORTED; }
     // Bands of about 24 MB of one operand (4 to 32 tiles).  Measured on [32768, 4096] x [6144, 4096]^T with bands of
     // row pairs: 12 (24 MB) 1409 TFLOP/s, 4: 1382, 8: 1404, 16: 1401, 23: 1385, 32: 1348 - the L2 serves both dies and
     // also carries the other operand and the stream of y, so far less than its 126 MB holds a band.  Bands of x
@@ -213,10 +339,44 @@ extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_
     const int64_t by_cols_traffic = w_bytes + x_bytes * ((gn + band - 1) / band);
     const int32_t by_cols = by_cols_traffic < by_rows_traffic ? 1 : 0;
     dim3 grid((unsigned)(2 * pairs), (unsigned)gn);           // clusters of two CTAs along x
-    lin::linear_kernel<<<grid, lin::kThreads, lin::kSmemBytes, static_cast<cudaStream_t>(cuda_stream)>>>(
-        tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, (int32_t)band, by_cols, status,
-        (long long)wait_limit_cycles(), test_skip_last_load());
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (rope)
+        lin::linear_kernel<true><<<grid, lin::kThreads, lin::kSmemBytes, stream>>>(
+            tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, (int32_t)band, by_cols, status,
+            (long long)wait_limit_cycles(), test_skip_last_load(), *rope);
+    else
+        lin::linear_kernel<false><<<grid, lin::kThreads, lin::kSmemBytes, stream>>>(
+            tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, (int32_t)band, by_cols, status,
+            (long long)wait_limit_cycles(), test_skip_last_load(), lin::Rope{});
     const cudaError_t err = cudaGetLastError();
-    if (err != cudaSuccess) { set_error("pec_linear: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
+    if (err != cudaSuccess) { set_error("%s: launch failed: %s", who, cudaGetErrorString(err)); return PEC_ERR_CUDA; }
+    return PEC_OK;
+}
+
+extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_t w_stride, void *y, int64_t y_stride,
+                          int64_t M, int32_t N, int32_t K, int32_t *status, void *cuda_stream)
+{
+    return linear_common("pec_linear", x, x_stride, w, w_stride, y, y_stride, M, N, K, status, cuda_stream, nullptr);
+}
+
+extern "C" int pec_linear_rope(const void *x, int64_t x_stride, const void *w, int64_t w_stride, void *y, int64_t y_stride,
+                               int64_t M, int32_t N, int32_t K, const float *rope_cos, const float *rope_sin, int64_t n_pos,
+                               const int32_t *positions, int64_t pos0, int32_t rot_cols, int32_t *status, void *cuda_stream)
+{
+    if (n_pos >= ((int64_t)1 << 31)) { set_error("pec_linear_rope: n_pos must be below 2^31"); return PEC_ERR_INVALID_ARG; }
+    lin::Rope rope = {rope_cos, rope_sin, positions, pos0, (int32_t)n_pos, rot_cols};
+    return linear_common("pec_linear_rope", x, x_stride, w, w_stride, y, y_stride, M, N, K, status, cuda_stream, &rope);
+}
+
+extern "C" int pec_rope_table(double theta, int64_t n_pos, int32_t D, float *cos_out, float *sin_out, void *cuda_stream)
+{
+    if (!cos_out || !sin_out || n_pos < 0 || !(theta > 0.0)) { set_error("pec_rope_table: need tables, n_pos >= 0 and theta > 0"); return PEC_ERR_INVALID_ARG; }
+    if (D != 128) { set_error("pec_rope_table: D must be 128"); return PEC_ERR_UNSUPPORTED; }
+    if (n_pos >= ((int64_t)1 << 31)) { set_error("pec_rope_table: n_pos must be below 2^31"); return PEC_ERR_INVALID_ARG; }
+    if (n_pos == 0) return PEC_OK;
+    const int64_t n = n_pos * 64;
+    lin::rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(std::log2(theta), n_pos, cos_out, sin_out);
+    const cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) { set_error("pec_rope_table: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;
 }

@@ -343,6 +343,53 @@ def test_attention_layer_steps_chain_through_strides(pec):
     assert np.abs(out.float().cpu().double().numpy() - oracle.linear(o.view(T, hq * 128).cpu(), w_l)).max() <= 2e-2
 
 
+def test_rope_table_matches_fp64_cos_and_sin(pec):
+    theta, n_pos = 500000.0, 70000
+    cos, sin = pec.pec_rope_table(theta, n_pos, DEV)
+    ang = np.arange(n_pos, dtype=np.float64)[:, None] * theta ** (-2.0 * np.arange(64, dtype=np.float64) / 128)[None, :]
+    assert np.abs(cos.cpu().double().numpy() - np.cos(ang)).max() <= 1e-7
+    assert np.abs(sin.cpu().double().numpy() - np.sin(ang)).max() <= 1e-7
+
+
+@pytest.mark.parametrize("M,N,K,rot,pos0", [(1, 128, 8, 128, 0), (130, 384, 72, 256, 5), (257, 6144, 512, 5120, 65000),
+                                            (600, 392, 64, 384, 499_000), (300, 256, 128, 0, 3)])
+def test_linear_rope_matches_oracle(pec, M, N, K, rot, pos0):
+    """Eq. 2 with the rotary encoding of the query and key heads in the GEMM's epilogue; rows are a chunk at pos0."""
+    theta = 500000.0
+    x = workloads.normal_tensor(18000 + M, 1, (M, K), torch.bfloat16)
+    w = (workloads.normal_tensor(18001 + N, 2, (N, K), torch.float32) / K ** 0.5).to(torch.bfloat16)
+    tables = pec.pec_rope_table(theta, pos0 + M, DEV)
+    y = pec.pec_linear_rope(x.to(DEV), w.to(DEV), tables, rot, pos0=pos0)
+    pec.check_status()
+    want = oracle.linear_rope(x, w, np.arange(pos0, pos0 + M), theta, rot)
+    err = np.abs(y.float().cpu().double().numpy() - want).max()
+    print(f"[parity] linear_rope {M}x{N}x{K} rot={rot} pos0={pos0}: max|dy| = {err:.3e}")
+    assert err <= 2e-2
+    if rot == 0:                                          # nothing to turn: the plain GEMM's bits
+        assert torch.equal(y, pec.pec_linear(x.to(DEV), w.to(DEV)))
+
+
+def test_linear_rope_packed_positions_and_attention_on_the_encoded_heads(pec):
+    """A packed batch: every row carries its position inside its own request; the encoded q and k then go through
+    the attention as strided slices, and each step is compared with the oracle applied to that step's inputs."""
+    lens, d, hq, hkv, theta = [300, 1, 515, 128], 256, 4, 2, 10000.0
+    cu = workloads.cu_seqlens(lens)
+    T = cu[-1]
+    pos = np.concatenate([np.arange(n) for n in lens]).astype(np.int32)
+    e = workloads.normal_tensor(18100, 1, (T, d), torch.bfloat16)
+    w_qkv = (workloads.normal_tensor(18101, 2, ((hq + 2 * hkv) * 128, d), torch.float32) / d ** 0.5).to(torch.bfloat16)
+    tables = pec.pec_rope_table(theta, max(lens), DEV)
+    qkv = pec.pec_linear_rope(e.to(DEV), w_qkv.to(DEV), tables, (hq + hkv) * 128, positions=torch.from_numpy(pos).to(DEV))
+    pec.check_status()
+    want = oracle.linear_rope(e, w_qkv, pos, theta, (hq + hkv) * 128)
+    assert np.abs(qkv.float().cpu().double().numpy() - want).max() <= 2e-2
+    fused = qkv.view(T, hq + 2 * hkv, 128)
+    q, k, v = fused[:, :hq], fused[:, hq:hq + hkv], fused[:, hq + hkv:]
+    o, lse = pec.pec_prefill_attn(q, k, v, cu_seqlens=torch.tensor(cu, dtype=torch.int32, device=DEV))
+    pec.check_status()
+    compare(o, lse, *oracle.varlen_attn(q.cpu(), k.cpu(), v.cpu(), cu), 2e-2, 1e-3, "attention on rotary-encoded q, k")
+
+
 def _random_partials(seed, rows, hq, n):
     """n fp32 partials with LSEs; about a fifth of the (row, head, part) entries empty (lse = -inf, o poisoned with NaN:
     an empty part must not be read), and a few rows empty in every part."""
