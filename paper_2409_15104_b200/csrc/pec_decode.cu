@@ -16,33 +16,70 @@
 
 namespace pec {
 
-constexpr int kReduceThreads = 128;                           // one thread per output channel
+constexpr int kReduceWarps = 8;
+constexpr int kReduceThreads = kReduceWarps * 32;
 
 // One CTA per query head: merges that head's partials over all slices.
 //   part_o [splits][g][Hkv][128] fp32, part_lse [splits][g][Hkv]; head = kvh * g + r.
+// A lane owns four channels; warp w takes slices w, w + 8, ... (their loads are independent, four in
+// flight per lane), the eight warps' sums meet in shared memory.  The maximum of the LSEs is found by
+// every warp for itself, one slice per lane at a time.
 template <bool kOutBf16>
 __global__ void __launch_bounds__(kReduceThreads)
 decode_reduce_kernel(const float *__restrict__ part_o, const float *__restrict__ part_lse, void *o, float *lse,
                      int splits, int g, int hkv)
 {
-    const int head = blockIdx.x, kvh = head / g, r = head % g, c = threadIdx.x;
+    __shared__ float4 sh_acc[kReduceWarps][32];
+    __shared__ float sh_tot[kReduceWarps];
+    const int head = blockIdx.x, kvh = head / g, r = head % g;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t item = (int64_t)r * hkv + kvh, stride = (int64_t)g * hkv;
+    // Launched as a programmatic dependent of the slice kernel: the launch itself overlaps that kernel's end, and
+    // nothing is read before the kernel has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     float m = -INFINITY;
-    for (int s = 0; s < splits; ++s) m = fmaxf(m, part_lse[s * stride + item]);
-    float tot = 0.f, acc = 0.f;
+    for (int s = lane; s < splits; s += 32) m = fmaxf(m, part_lse[s * stride + item]);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+    float tot = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (m != -INFINITY) {
-        for (int s = 0; s < splits; ++s) {
+#pragma unroll 4
+        for (int s = warp; s < splits; s += kReduceWarps) {
             const float l = part_lse[s * stride + item];
-            if (l == -INFINITY) continue;                     // empty slice: its O is not read
-            const float w = expf(l - m);
-            tot += w;
-            acc = fmaf(w, part_o[(s * stride + item) * kHeadDim + c], acc);
+            const float w = (l == -INFINITY) ? 0.f : __expf(l - m);
+            if (w != 0.f) {                                   // empty slice: its O is not used
+                const float4 v = *reinterpret_cast<const float4 *>(part_o + (s * stride + item) * kHeadDim + 4 * lane);
+                acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y); acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+                tot += w;
+            }
         }
-        acc /= tot;
     }
-    if (kOutBf16) static_cast<__nv_bfloat16 *>(o)[(int64_t)head * kHeadDim + c] = __float2bfloat16_rn(acc);
-    else          static_cast<float *>(o)[(int64_t)head * kHeadDim + c] = acc;
-    if (c == 0) lse[head] = (m == -INFINITY) ? -INFINITY : m + logf(tot);
+    sh_acc[warp][lane] = acc;
+    if (lane == 0) sh_tot[warp] = tot;
+    __syncthreads();
+    if (warp == 0) {
+        tot = 0.f;
+        acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int w = 0; w < kReduceWarps; ++w) {
+            const float4 v = sh_acc[w][lane];
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            tot += sh_tot[w];
+        }
+        const float inv = tot > 0.f ? 1.f / tot : 0.f;
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+        if (kOutBf16) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+            uint2 pk;
+            pk.x = *reinterpret_cast<uint32_t *>(&lo);
+            pk.y = *reinterpret_cast<uint32_t *>(&hi);
+            *reinterpret_cast<uint2 *>(static_cast<__nv_bfloat16 *>(o) + (int64_t)head * kHeadDim + 4 * lane) = pk;
+        } else {
+            *reinterpret_cast<float4 *>(static_cast<float *>(o) + (int64_t)head * kHeadDim + 4 * lane) = acc;
+        }
+        if (lane == 0) lse[head] = (m == -INFINITY) ? -INFINITY : m + logf(tot);
+    }
 }
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -127,10 +164,18 @@ static int run_decode(const pec_decode_args *a, const DecodeShape &shape, void *
     p.split_keys = shape.split_keys;
     const int rc = launch_attn_split_bf16(p, stream);
     if (rc != PEC_OK) return rc;
-    if (a->o_dtype == PEC_BF16)
-        decode_reduce_kernel<true><<<a->Hq, kReduceThreads, 0, stream>>>(part_o, part_lse, a->o, a->lse, shape.splits, g, a->Hkv);
-    else
-        decode_reduce_kernel<false><<<a->Hq, kReduceThreads, 0, stream>>>(part_o, part_lse, a->o, a->lse, shape.splits, g, a->Hkv);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)a->Hq);
+    cfg.blockDim = dim3(kReduceThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float *po = part_o, *pl = part_lse;
+    if (a->o_dtype == PEC_BF16) cudaLaunchKernelEx(&cfg, decode_reduce_kernel<true>, po, pl, a->o, a->lse, (int)shape.splits, g, (int)a->Hkv);
+    else                        cudaLaunchKernelEx(&cfg, decode_reduce_kernel<false>, po, pl, a->o, a->lse, (int)shape.splits, g, (int)a->Hkv);
     const cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("%s: launch failed: %s", who, cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;
