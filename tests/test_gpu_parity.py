@@ -692,3 +692,57 @@ def test_launches_that_overlap_their_predecessor_give_the_same_bits(pec):
         pec.check_status()
         assert torch.equal(o, base[0]) and torch.equal(lse, base[1])
     compare(o, lse, *oracle.prefill_attn(q, k, v, seq_len=S), *TOL[torch.bfloat16], "overlapping chain")
+
+
+# ------------------------------------------------------------------ many random calls, the two kernels against each other
+def test_many_random_calls_bf16_kernel_against_fp32_kernel(pec):
+    """A cross-check beside the oracle comparisons above, not instead of them: 600 seeded calls (lengths to 9000, chunks,
+    prefixes, key partitions, query partitions, incoming state, fused-QKV strides, score scales, moved maxima) through the
+    tensor-core kernel and through the fp32 kernel (itself compared with the oracle in full elsewhere) on the same
+    inputs; every element of O and LSE must agree and the same rows must be empty."""
+    worst_o = worst_l = 0.0
+    for seed in range(600):
+        g = np.random.Generator(np.random.Philox(key=777000 + seed))
+        S = int(g.integers(1, 9000)) if seed % 3 else int(g.integers(1, 700))
+        hkv = int(g.choice([1, 2, 3]))
+        hq = hkv * int(g.choice([1, 2, 4, 8]))
+        P = int(g.choice([1, 1, 2, 3, 4, 8, 16]))
+        align = int(g.choice([1, 16, 64, 128, 256]))
+        causal = bool(g.integers(0, 5) > 0)
+        c0 = int(g.integers(0, S)) if g.integers(0, 2) else 0
+        n = int(g.integers(1, S - c0 + 1)) if g.integers(0, 2) else S - c0
+        kv_len = int(g.integers(c0 + n, S + 1)) if causal else int(g.integers(1, S + 1))
+        part = int(g.integers(0, P))
+        qP = int(g.choice([0, 0, 2, 3, 4])) if causal else 0
+        qp = int(g.integers(0, qP)) if qP else 0
+        use_acc = bool(g.integers(0, 2)) and P > 1
+        fused_layout = bool(g.integers(0, 2))
+        scale = float(g.choice([0.0, 0.05, 0.2]))
+        gen = torch.Generator(device=DEV).manual_seed(seed)
+        buf = torch.randn(S, hq + 2 * hkv, 128, device=DEV, generator=gen).to(torch.bfloat16)
+        if seed % 4 == 0:
+            buf[:: max(1, S // 7), hq:hq + hkv] *= 4                   # keys that move the running maximum
+        q, k, v = buf[:, :hq], buf[:, hq:hq + hkv], buf[:, hq + hkv:]
+        if not fused_layout:
+            q, k, v = q.contiguous(), k.contiguous(), v.contiguous()
+        qf, kf, vf = q.float().contiguous(), k.float().contiguous(), v.float().contiguous()
+        kw = dict(seq_len=S, chunk_start=c0, chunk_len=n, kv_len=kv_len, part_id=part, num_parts=P, part_align=align,
+                  causal=causal, softmax_scale=scale, q_part_id=qp, q_num_parts=qP)
+        o32 = torch.zeros(n, hq, 128, device=DEV); l32 = torch.full((n, hq), float("-inf"), device=DEV)
+        acc32 = acc16 = None
+        if use_acc:                                                    # state: the fp32 kernel's result over another partition
+            pec.pec_prefill_attn(qf, kf, vf, o=o32, lse=l32, **{**kw, "part_id": (part + 1) % P})
+            acc32, acc16 = (o32.clone(), l32.clone()), (o32.clone(), l32.clone())
+        o16, l16 = o32.clone(), l32.clone()
+        pec.pec_prefill_attn(qf, kf, vf, o=o32, lse=l32, acc=acc32, **kw)
+        pec.pec_prefill_attn(q, k, v, o=o16, lse=l16, acc=acc16, **kw)
+        pec.check_status()
+        what = f"seed {seed}: S={S} hq={hq} hkv={hkv} P={P} part={part} align={align} causal={causal} c0={c0} n={n} kv={kv_len} qP={qP} qp={qp} acc={use_acc} fused={fused_layout} scale={scale}"
+        fin = torch.isfinite(l32)
+        assert not torch.isnan(o16).any() and not torch.isnan(l16).any(), what
+        assert torch.equal(torch.isfinite(l16), fin), what
+        eo = float((o16 - o32).abs().max())
+        el = float((l16[fin] - l32[fin]).abs().max()) if fin.any() else 0.0
+        assert eo <= 2e-2 * max(1.0, float(o32.abs().max()) / 4) and el <= 1e-3, what
+        worst_o, worst_l = max(worst_o, eo), max(worst_l, el)
+    print(f"[cross-check] 600 random calls, bf16 against fp32 kernel: max|dO| = {worst_o:.3e}, max|dLSE| = {worst_l:.3e}")
