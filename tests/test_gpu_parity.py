@@ -746,3 +746,56 @@ def test_many_random_calls_bf16_kernel_against_fp32_kernel(pec):
         assert eo <= 2e-2 * max(1.0, float(o32.abs().max()) / 4) and el <= 1e-3, what
         worst_o, worst_l = max(worst_o, eo), max(worst_l, el)
     print(f"[cross-check] 600 random calls, bf16 against fp32 kernel: max|dO| = {worst_o:.3e}, max|dLSE| = {worst_l:.3e}")
+
+
+def test_many_random_packed_batches_with_and_without_the_worklist(pec):
+    """200 seeded packed batches (1-39 requests of 0-1199 rows, now and then one of several thousand): the work-list
+    changes the order of the tiles and nothing else (identical bits), and every element agrees with the fp32 kernel."""
+    from paper_2409_15104_b200 import prefill
+    worst_o = worst_l = 0.0
+    for seed in range(200):
+        g = np.random.Generator(np.random.Philox(key=888000 + seed))
+        B = int(g.integers(1, 40))
+        lens = [int(x) for x in g.integers(0, 1200, size=B)]
+        if seed % 5 == 0:
+            lens[int(g.integers(0, B))] = int(g.integers(2000, 6000))
+        cu = [0] + [int(x) for x in np.cumsum(lens)]
+        if cu[-1] == 0:
+            continue
+        hkv = int(g.choice([1, 2]))
+        hq = hkv * int(g.choice([1, 4, 8]))
+        gen = torch.Generator(device=DEV).manual_seed(seed)
+        buf = torch.randn(cu[-1], hq + 2 * hkv, 128, device=DEV, generator=gen).to(torch.bfloat16)
+        q, k, v = buf[:, :hq], buf[:, hq:hq + hkv], buf[:, hq + hkv:]
+        dcu = torch.tensor(cu, dtype=torch.int32, device=DEV)
+        o1, l1 = prefill.varlen_prefill(q, k, v, dcu)
+        o2, l2 = prefill.varlen_prefill(q, k, v, dcu, worklist=prefill.make_worklist(cu, torch.bfloat16, DEV))
+        o3, l3 = pec.pec_prefill_attn(q.float().contiguous(), k.float().contiguous(), v.float().contiguous(), cu_seqlens=dcu)
+        pec.check_status()
+        what = f"seed {seed}: lens={lens} hq={hq} hkv={hkv}"
+        assert torch.equal(o1, o2) and torch.equal(l1, l2), what
+        assert not torch.isnan(o1).any() and not torch.isnan(l1).any(), what
+        eo, el = float((o1.float() - o3).abs().max()), float((l1 - l3).abs().max())
+        assert eo <= 2.5e-2 and el <= 1e-3, what             # the bf16 output's own rounding on top of 2e-2
+        worst_o, worst_l = max(worst_o, eo), max(worst_l, el)
+    print(f"[cross-check] 200 random packed batches, bf16 against fp32 kernel: max|dO| = {worst_o:.3e}, max|dLSE| = {worst_l:.3e}")
+
+
+def test_many_random_decode_calls_match_oracle(pec):
+    """60 seeded decode calls: cache lengths to 20000, key ranges inside the cache (empty ones too), 1-16 query heads
+    per KV head, slice counts given or chosen by the library."""
+    for seed in range(60):
+        g = np.random.Generator(np.random.Philox(key=999000 + seed))
+        L = int(g.integers(1, 20000))
+        hkv = int(g.choice([1, 2, 8]))
+        grp = int(g.choice([1, 2, 4, 8, 16]))
+        lo = int(g.integers(0, L)) if g.integers(0, 2) else 0
+        hi = int(g.integers(lo, L + 1)) if g.integers(0, 2) else L
+        splits = int(g.choice([0, 0, 1, 2, 3, 7, 16, 37]))
+        k = workloads.normal_tensor(30000 + seed, 2, (L, hkv, 128), torch.bfloat16)
+        v = workloads.normal_tensor(30000 + seed, 3, (L, hkv, 128), torch.bfloat16)
+        q = workloads.normal_tensor(30000 + seed, 1, (hkv * grp, 128), torch.bfloat16)
+        o, lse = pec.pec_decode_attn(q.to(DEV), k.to(DEV), v.to(DEV), kv_lo=lo, kv_hi=hi, num_splits=splits)
+        pec.check_status()
+        want = oracle.attn_rows(q[None], [L - 1], k, v, [(lo, hi)] if hi > lo else [], False)
+        compare(o[None], lse[None], *want, 2e-2, 1e-3, f"decode seed {seed}: L={L} keys [{lo},{hi}) {hkv * grp}/{hkv} heads splits={splits}")
