@@ -396,24 +396,30 @@ int pec_linear(const void *x, int64_t x_stride, const void *w, int64_t w_stride,
  *     y'[i]      = y[i] cos(a) - y[i + 64] sin(a)
  *     y'[i + 64] = y[i + 64] cos(a) + y[i] sin(a),      a = p * theta^(-2 i / 128).
  * Columns from rot_cols on (the value heads) are left as they are.  rot_cols: multiple of 128, <= N.
- * rope_cos / rope_sin: device [n_pos, 64] fp32 tables of cos(a) and sin(a) (pec_rope_table fills
- * them), 16-byte aligned.  Row r is at position positions[r] (device int32 [M], e.g. a packed
- * batch's positions within their requests) or, with positions == NULL, at pos0 + r (a chunk of one
- * request, Section 5.1); positions outside [0, n_pos) are clamped to the table's ends, and the
- * host rejects pos0 + M > n_pos.  Everything else as in pec_linear.
+ * rope_table: device table for positions 0 .. n_pos - 1, pec_rope_table_floats(n_pos) floats filled
+ * by pec_rope_table, 16-byte aligned.  Row r is at position positions[r] (device int32 [M], e.g. a
+ * packed batch's positions within their requests) or, with positions == NULL, at pos0 + r (a chunk
+ * of one request, Section 5.1); positions outside [0, n_pos) are clamped to the table's ends, and
+ * the host rejects pos0 + M > n_pos.  Everything else as in pec_linear.
  * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.
  */
 int pec_linear_rope(const void *x, int64_t x_stride, const void *w, int64_t w_stride, void *y, int64_t y_stride,
-                    int64_t M, int32_t N, int32_t K, const float *rope_cos, const float *rope_sin, int64_t n_pos,
+                    int64_t M, int32_t N, int32_t K, const float *rope_table, int64_t n_pos,
                     const int32_t *positions, int64_t pos0, int32_t rot_cols, int32_t *status, void *cuda_stream);
 
 /*
- * Fills the tables pec_linear_rope reads: cos_out[p][i] = cos(p * theta^(-2 i / D)),
- * sin_out[p][i] likewise, for 0 <= p < n_pos, 0 <= i < D / 2, worked out in fp64 on the device
- * and stored as fp32 (device [n_pos, D / 2] each).  D must be 128; theta > 0 (500000 for Llama-3).
- * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ * The table pec_linear_rope reads, for positions 0 .. n_pos - 1 and D = 128.  The angle of position
+ * p = 64 a + b and channel i is split by the addition theorem,
+ *     cos(p f_i) = C[a][i] F[i][b] - S[a][i] G[i][b],   sin(p f_i) = S[a][i] F[i][b] + C[a][i] G[i][b],
+ *     f_i = theta^(-2 i / D),  C, S = cos, sin(64 a f_i),  F, G = cos, sin(b f_i),
+ * so that the kernel's reads are small and contiguous.  Layout, in floats:
+ * F [64][64] | G [64][64] | C [na][64] | S [na][64] with na = ceil(n_pos / 64); every entry is worked
+ * out in fp64 on the device and stored as fp32.  pec_rope_table_floats returns the table's length
+ * (0 for a negative or too large n_pos); theta > 0 (500000 for Llama-3).
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.
  */
-int pec_rope_table(double theta, int64_t n_pos, int32_t D, float *cos_out, float *sin_out, void *cuda_stream);
+size_t pec_rope_table_floats(int64_t n_pos);
+int pec_rope_table(double theta, int64_t n_pos, int32_t D, float *table, void *cuda_stream);
 
 /*
  * The post-self-attention linear layer (Eq. 5) taking partial attention results as they are:
@@ -425,8 +431,8 @@ int pec_rope_table(double theta, int64_t n_pos, int32_t D, float *cos_out, float
  * n key partitions (Section 2.2).
  * o_parts / lse_parts: HOST arrays of n DEVICE pointers (1 <= n <= PEC_LINEAR_MERGED_MAX_PARTS),
  * [rows, Hq, D] fp32 and [rows, Hq] fp32, contiguous, o 16-byte aligned; the arrays are read
- * during the call only.  A part whose lse is -inf for a (row, head) is not read there; where
- * every part's is, the merged row is 0.  D must be 128; the contraction runs over K = Hq * D.
+ * during the call only.  What a part holds where its lse is -inf is not used (it may be anything,
+ * NaN included); where every part's lse is -inf the merged row is 0.  D must be 128; the contraction runs over K = Hq * D.
  * w: device [N, K] bf16, y: device [rows, N] bf16; row strides in elements (multiples of 8),
  * 16-byte aligned; N a multiple of 8.  `status`: required device word, used as in pec_attn_args.
  * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.

@@ -94,7 +94,7 @@ class pec_plan(ctypes.Structure):
 EXPORTS = ("pec_prefill_attn", "pec_workspace_size", "pec_attn_merge", "pec_attn_merge_n", "pec_plan_partitions",
            "pec_last_error", "pec_decode_attn", "pec_decode_workspace_size", "pec_decode_attn_static", "pec_select_sp", "pec_linear",
            "pec_plan_ring", "pec_balance_batches", "pec_plan_worklist", "pec_worklist_block_m", "pec_control",
-           "pec_linear_merged", "pec_linear_rope", "pec_rope_table")
+           "pec_linear_merged", "pec_linear_rope", "pec_rope_table", "pec_rope_table_floats")
 PEC_CTL_WAIT_LIMIT_CYCLES, PEC_CTL_TEST_SKIP_LAST_LOAD = 1, 2
 PEC_DECODE_STATIC_SCRATCH_BYTES = 4 * 1024 * 1024
 PEC_MERGE_MAX_PARTS = 16
@@ -137,11 +137,12 @@ def load():
     lib.pec_linear_rope.restype = ctypes.c_int
     lib.pec_linear_rope.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
                                     ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
-                                    ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32,
+                                    ctypes.c_int64, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32,
                                     ctypes.c_void_p, ctypes.c_void_p]
     lib.pec_rope_table.restype = ctypes.c_int
-    lib.pec_rope_table.argtypes = [ctypes.c_double, ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
-                                   ctypes.c_void_p]
+    lib.pec_rope_table.argtypes = [ctypes.c_double, ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
+    lib.pec_rope_table_floats.restype = ctypes.c_size_t
+    lib.pec_rope_table_floats.argtypes = [ctypes.c_int64]
     lib.pec_linear_merged.restype = ctypes.c_int
     lib.pec_linear_merged.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p), ctypes.c_int32,
                                       ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int64,
@@ -383,11 +384,24 @@ def pec_linear(x, w, y=None, stream=None):
 
 
 def pec_rope_table(theta, n_pos, device, stream=None):
-    """(cos, sin) tables [n_pos, 64] fp32 of the rotary position encoding for head_dim 128."""
+    """The rotary-encoding table for positions 0 .. n_pos - 1 (head_dim 128): (tensor, n_pos), as pec_linear_rope takes it."""
     lib = load()
-    cos = torch.empty((n_pos, 64), dtype=torch.float32, device=device)
-    sin = torch.empty((n_pos, 64), dtype=torch.float32, device=device)
-    _check(lib.pec_rope_table(float(theta), n_pos, 128, cos.data_ptr(), sin.data_ptr(), _stream_ptr(stream)))
+    table = torch.empty((lib.pec_rope_table_floats(n_pos),), dtype=torch.float32, device=device)
+    _check(lib.pec_rope_table(float(theta), n_pos, 128, table.data_ptr(), _stream_ptr(stream)))
+    return table, n_pos
+
+
+def rope_table_angles(tables):
+    """(cos, sin) [n_pos, 64] in fp64 as the kernel combines them from the table's fp32 entries (for inspection and tests)."""
+    table, n_pos = tables
+    t = table.double().cpu()
+    na = (n_pos + 63) // 64
+    F, G = t[:4096].view(64, 64), t[4096:8192].view(64, 64)            # [i][b]
+    C, S = t[8192:8192 + na * 64].view(na, 64), t[8192 + na * 64:].view(na, 64)
+    p = torch.arange(n_pos)
+    a, b = p // 64, p % 64
+    cos = C[a] * F.T[b] - S[a] * G.T[b]
+    sin = S[a] * F.T[b] + C[a] * G.T[b]
     return cos, sin
 
 
@@ -395,10 +409,10 @@ def pec_linear_rope(x, w, tables, rot_cols, *, positions=None, pos0=0, y=None, s
     """y = x w^T with the rotary encoding of the leading rot_cols columns (whole heads of 128); tables = pec_rope_table(...).
     positions: int32 CUDA tensor [M] (packed batches) or None: row r is at position pos0 + r."""
     lib = load()
-    cos, sin = tables
+    table, n_pos = tables
     assert x.is_cuda and w.is_cuda and x.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
     assert x.stride(1) == 1 and w.stride(1) == 1 and x.shape[1] == w.shape[1]
-    assert cos.is_contiguous() and sin.is_contiguous() and cos.shape == sin.shape and cos.shape[1] == 64
+    assert table.is_cuda and table.is_contiguous() and table.dtype == torch.float32
     M, K = x.shape
     N = w.shape[0]
     if y is None:
@@ -407,9 +421,8 @@ def pec_linear_rope(x, w, tables, rot_cols, *, positions=None, pos0=0, y=None, s
     if positions is not None:
         assert positions.is_cuda and positions.dtype == torch.int32 and positions.is_contiguous() and positions.numel() == M
     _check(lib.pec_linear_rope(x.data_ptr(), x.stride(0), w.data_ptr(), w.stride(0), y.data_ptr(), y.stride(0), M, N, K,
-                               cos.data_ptr(), sin.data_ptr(), cos.shape[0],
-                               positions.data_ptr() if positions is not None else None, pos0, rot_cols,
-                               status_word(x.device).data_ptr(), _stream_ptr(stream)))
+                               table.data_ptr(), n_pos, positions.data_ptr() if positions is not None else None, pos0,
+                               rot_cols, status_word(x.device).data_ptr(), _stream_ptr(stream)))
     return y
 
 

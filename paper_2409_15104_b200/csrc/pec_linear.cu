@@ -47,13 +47,20 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Wa
 
 // Rotary position encoding applied to the accumulator before it is rounded (kRope): the leading rot_cols
 // columns of y are heads of 128 channels; channel i < 64 of a head pairs with channel i + 64 and the pair of
-// the row at position p is turned by the angle whose cosine and sine are cos_tab[p][i], sin_tab[p][i].
+// the row at position p is turned by the angle p * f_i.  The angle's cosine and sine come from two small tables
+// by the addition theorem, p = 64 a + b:  cos(p f) = C[a][i] F[i][b] - S[a][i] G[i][b], sin likewise, with
+// C, S = cos, sin(64 a f_i) ("coarse", one row of 64 per 64 positions) and F, G = cos, sin(b f_i) ("fine",
+// 64 x 64, stored channel-major so that a warp's 32 consecutive positions read 128 contiguous bytes).
+// A table of every position's angles read row by row costs 32 memory wavefronts per load instruction (each
+// lane its own line) and made the epilogue 6 % of the GEMM; these reads are one or two wavefronts each.
+// Table layout (floats): F [64][64] | G [64][64] | C [na][64] | S [na][64], na = ceil(n_pos / 64).
 struct Rope {
-    const float *cos_tab, *sin_tab;                           // [n_pos, 64] fp32
+    const float *table;
     const int32_t *positions;                                 // [M] or NULL: row r is at position pos0 + r
     int64_t pos0;
     int32_t n_pos, rot_cols;
 };
+constexpr int kRopeFine = 64 * 64;
 
 // 32 accumulator columns -> bf16, 16 bytes per store, columns at or past N left out.
 __device__ __forceinline__ void store_chunk(__nv_bfloat16 *dst, const uint32_t (&r)[32], int col0, int32_t N)
@@ -85,13 +92,20 @@ __device__ __forceinline__ void store_chunk16(__nv_bfloat16 *dst, const uint32_t
         }
     }
 }
-// Sixteen cosines and sines of a row, channels i0 .. i0 + 15 (row[0] = its line of the cosine table, row[1] of the sines).
-__device__ __forceinline__ void rope_fetch(const float *const (&row)[2], int i0, float4 (&c)[4], float4 (&s)[4])
+// Cosines and sines of sixteen channels i0 .. i0 + 15 for the row at position 64 a + b (see Rope).
+__device__ __forceinline__ void rope_angles(const float *table, int na, int a, int b, int i0, float (&c)[16], float (&s)[16])
 {
+    const float *cc = table + 2 * kRopeFine + (int64_t)a * 64 + i0, *cs = cc + (int64_t)na * 64;
+    float4 c4[4], s4[4];
 #pragma unroll
-    for (int v = 0; v < 4; ++v) {
-        c[v] = __ldg(reinterpret_cast<const float4 *>(row[0] + i0) + v);
-        s[v] = __ldg(reinterpret_cast<const float4 *>(row[1] + i0) + v);
+    for (int v = 0; v < 4; ++v) { c4[v] = __ldg(reinterpret_cast<const float4 *>(cc) + v); s4[v] = __ldg(reinterpret_cast<const float4 *>(cs) + v); }
+    const float *ccf = reinterpret_cast<const float *>(c4), *csf = reinterpret_cast<const float *>(s4);
+    const float *f = table + i0 * 64 + b, *g = f + kRopeFine;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const float fc = __ldg(f + j * 64), fs = __ldg(g + j * 64);
+        c[j] = ccf[j] * fc - csf[j] * fs;
+        s[j] = csf[j] * fc + ccf[j] * fs;
     }
 }
 // Two 16-column accumulator loads in flight, then one wait.
@@ -202,15 +216,12 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
         __syncwarp();
     } else {
         const int64_t row = m0 + warp * 32 + lane;
-        [[maybe_unused]] const float *rope_row[2] = {nullptr, nullptr};
-        [[maybe_unused]] float4 c_next[4], s_next[4];
+        [[maybe_unused]] int rope_a = 0, rope_b = 0, rope_na = 0;
         if constexpr (kRope) {
             int64_t pos = 0;
             if (row < M) pos = rope.positions ? (int64_t)rope.positions[row] : rope.pos0 + row;
             pos = pos < 0 ? 0 : (pos >= rope.n_pos ? rope.n_pos - 1 : pos);
-            rope_row[0] = rope.cos_tab + pos * 64;
-            rope_row[1] = rope.sin_tab + pos * 64;
-            if (n0 < rope.rot_cols) rope_fetch(rope_row, 0, c_next, s_next);     // a tile of value heads needs none
+            rope_a = (int)(pos >> 6); rope_b = (int)(pos & 63); rope_na = (rope.n_pos + 63) >> 6;
         }
         const bool ok = __all_sync(0xffffffffu, n_kb == 0 || wait_bar(smem_u32(&sh->acc_full), 0, wctx));
         if (ok) {
@@ -225,16 +236,12 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
                 }
             } else {
                 // The tile's 256 columns are two heads; a thread holds a whole row, so both channels of a pair are its own.
-                // Sixteen pairs of both heads per step, so a row's cosines and sines are fetched once per tile; those of a
-                // step are asked for one step ahead (those of the first step before the wait for the accumulator).
+                // Sixteen pairs of both heads per step, so a row's cosines and sines are worked out once per tile.
                 const bool turn0 = n0 < rope.rot_cols, turn1 = n0 + 128 < rope.rot_cols;    // rot_cols: whole heads
 #pragma unroll 1
                 for (int it = 0; it < 4; ++it) {              // channels 16 it .. 16 it + 15 and their partners, both heads
-                    float4 c4[4], s4[4];
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) { c4[v] = c_next[v]; s4[v] = s_next[v]; }
-                    if (it < 3 && turn0) rope_fetch(rope_row, (it + 1) * 16, c_next, s_next);
-                    const float *cf = reinterpret_cast<const float *>(c4), *sf = reinterpret_cast<const float *>(s4);
+                    float cf[16], sf[16];
+                    if (turn0) rope_angles(rope.table, rope_na, rope_a, rope_b, it * 16, cf, sf);   // a tile of value heads needs none
 #pragma unroll
                     for (int hh = 0; hh < 2; ++hh) {
                         const int col_a = hh * 128 + it * 16, col_b = col_a + 64;
@@ -266,19 +273,28 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
 }  // namespace lin
 }  // namespace pec
 
-// cos and sin of position * theta^(-2 i / 128), i < 64, worked out in fp64 and stored as fp32.
+// The two-level tables of Rope, worked out in fp64 and stored as fp32: one thread per (fine or coarse) entry.
 namespace pec {
 namespace lin {
-__global__ void rope_table_kernel(double log2_theta, int64_t n_pos, float *cos_out, float *sin_out)
+__global__ void rope_table_kernel(double log2_theta, int64_t na, float *table)
 {
     const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= n_pos * 64) return;
-    const int i = (int)(idx & 63);
-    const double inv_freq = exp2(-(double)(2 * i) / 128.0 * log2_theta);
+    if (idx >= kRopeFine + na * 64) return;
+    int i;
+    double p;
+    float *c_out, *s_out;
+    if (idx < kRopeFine) {                                    // fine: channel-major, F[i][b]
+        i = (int)(idx >> 6); p = (double)(idx & 63);
+        c_out = table + idx; s_out = c_out + kRopeFine;
+    } else {                                                  // coarse: C[a][i]
+        const int64_t j = idx - kRopeFine;
+        i = (int)(j & 63); p = (double)((j >> 6) * 64);
+        c_out = table + 2 * kRopeFine + j; s_out = c_out + na * 64;
+    }
     double s, c;
-    sincos((double)(idx >> 6) * inv_freq, &s, &c);
-    cos_out[idx] = (float)c;
-    sin_out[idx] = (float)s;
+    sincos(p * exp2(-(double)(2 * i) / 128.0 * log2_theta), &s, &c);
+    *c_out = (float)c;
+    *s_out = (float)s;
 }
 }  // namespace lin
 }  // namespace pec
@@ -298,16 +314,15 @@ static int linear_common(const char *who, const void *x, int64_t x_stride, const
         return PEC_ERR_ALIGNMENT;
     }
     if (rope) {
-        if (!rope->cos_tab || !rope->sin_tab || rope->n_pos < 1) { set_error("%s: the cos / sin tables must be non-NULL with n_pos >= 1", who); return PEC_ERR_INVALID_ARG; }
+        if (!rope->table || rope->n_pos < 1) { set_error("%s: the table must be non-NULL with n_pos >= 1", who); return PEC_ERR_INVALID_ARG; }
         if (rope->rot_cols < 0 || rope->rot_cols > N) { set_error("%s: rot_cols must lie in [0, N]", who); return PEC_ERR_INVALID_ARG; }
         if (rope->rot_cols % 128 != 0) { set_error("%s: rot_cols must be a multiple of 128 (whole heads)", who); return PEC_ERR_UNSUPPORTED; }
         if (!rope->positions && (rope->pos0 < 0 || rope->pos0 + M > rope->n_pos)) {
             set_error("%s: positions pos0 .. pos0 + M - 1 must lie inside the tables", who);
             return PEC_ERR_INVALID_ARG;
         }
-        if ((reinterpret_cast<uintptr_t>(rope->cos_tab) & 15u) || (reinterpret_cast<uintptr_t>(rope->sin_tab) & 15u) ||
-            (reinterpret_cast<uintptr_t>(rope->positions) & 3u)) {
-            set_error("%s: the cos / sin tables must be 16-byte aligned", who);
+        if ((reinterpret_cast<uintptr_t>(rope->table) & 15u) || (reinterpret_cast<uintptr_t>(rope->positions) & 3u)) {
+            set_error("%s: the table must be 16-byte aligned", who);
             return PEC_ERR_ALIGNMENT;
         }
     }
@@ -360,22 +375,28 @@ extern "C" int pec_linear(const void *x, int64_t x_stride, const void *w, int64_
 }
 
 extern "C" int pec_linear_rope(const void *x, int64_t x_stride, const void *w, int64_t w_stride, void *y, int64_t y_stride,
-                               int64_t M, int32_t N, int32_t K, const float *rope_cos, const float *rope_sin, int64_t n_pos,
+                               int64_t M, int32_t N, int32_t K, const float *rope_table, int64_t n_pos,
                                const int32_t *positions, int64_t pos0, int32_t rot_cols, int32_t *status, void *cuda_stream)
 {
     if (n_pos >= ((int64_t)1 << 31)) { set_error("pec_linear_rope: n_pos must be below 2^31"); return PEC_ERR_INVALID_ARG; }
-    lin::Rope rope = {rope_cos, rope_sin, positions, pos0, (int32_t)n_pos, rot_cols};
+    lin::Rope rope = {rope_table, positions, pos0, (int32_t)n_pos, rot_cols};
     return linear_common("pec_linear_rope", x, x_stride, w, w_stride, y, y_stride, M, N, K, status, cuda_stream, &rope);
 }
 
-extern "C" int pec_rope_table(double theta, int64_t n_pos, int32_t D, float *cos_out, float *sin_out, void *cuda_stream)
+extern "C" size_t pec_rope_table_floats(int64_t n_pos)
 {
-    if (!cos_out || !sin_out || n_pos < 0 || !(theta > 0.0)) { set_error("pec_rope_table: need tables, n_pos >= 0 and theta > 0"); return PEC_ERR_INVALID_ARG; }
+    if (n_pos < 0 || n_pos >= ((int64_t)1 << 31)) return 0;
+    return (size_t)(2 * lin::kRopeFine) + (size_t)((n_pos + 63) / 64) * 128;
+}
+
+extern "C" int pec_rope_table(double theta, int64_t n_pos, int32_t D, float *table, void *cuda_stream)
+{
+    if (!table || n_pos < 0 || !(theta > 0.0)) { set_error("pec_rope_table: need a table, n_pos >= 0 and theta > 0"); return PEC_ERR_INVALID_ARG; }
     if (D != 128) { set_error("pec_rope_table: D must be 128"); return PEC_ERR_UNSUPPORTED; }
     if (n_pos >= ((int64_t)1 << 31)) { set_error("pec_rope_table: n_pos must be below 2^31"); return PEC_ERR_INVALID_ARG; }
-    if (n_pos == 0) return PEC_OK;
-    const int64_t n = n_pos * 64;
-    lin::rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(std::log2(theta), n_pos, cos_out, sin_out);
+    if (reinterpret_cast<uintptr_t>(table) & 15u) { set_error("pec_rope_table: the table must be 16-byte aligned"); return PEC_ERR_ALIGNMENT; }
+    const int64_t na = (n_pos + 63) / 64, n = lin::kRopeFine + na * 64;
+    lin::rope_table_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(std::log2(theta), na, table);
     const cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("pec_rope_table: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;

@@ -169,22 +169,24 @@ def test_decode_validates_on_the_host_and_sizes_its_workspace():
 
 def test_linear_rope_and_table_validate_on_the_host():
     lib = binding.load()
-    ok = dict(x=4096, xs=64, w=8192, ws=64, y=12288, ys=256, M=10, N=256, K=64, c=65536, s=131072, npos=100, pos=None, pos0=0,
+    ok = dict(x=4096, xs=64, w=8192, ws=64, y=12288, ys=256, M=10, N=256, K=64, t=65536, npos=100, pos=None, pos0=0,
               rot=128, st=16384)
 
     def call(**over):
         a = {**ok, **over}
-        return lib.pec_linear_rope(a["x"], a["xs"], a["w"], a["ws"], a["y"], a["ys"], a["M"], a["N"], a["K"], a["c"], a["s"],
+        return lib.pec_linear_rope(a["x"], a["xs"], a["w"], a["ws"], a["y"], a["ys"], a["M"], a["N"], a["K"], a["t"],
                                    a["npos"], a["pos"], a["pos0"], a["rot"], a["st"], None)
 
     assert call(M=0) == 0
-    assert call(c=None) == -1 and call(s=None) == -1 and call(npos=0) == -1 and call(x=None) == -1
+    assert call(t=None) == -1 and call(npos=0) == -1 and call(x=None) == -1
     assert call(rot=384) == -1 and call(rot=-128) == -1 and call(pos0=91) == -1 and call(pos0=-1) == -1
     assert call(rot=64) == -2 and call(N=260, ys=264) == -2
-    assert call(c=65540) == -3 and call(pos=2050) == -3
-    assert lib.pec_rope_table(500000.0, 0, 128, 4096, 8192, None) == 0
-    assert lib.pec_rope_table(500000.0, 10, 64, 4096, 8192, None) == -2
-    assert lib.pec_rope_table(0.0, 10, 128, 4096, 8192, None) == -1 and lib.pec_rope_table(1e4, 10, 128, None, 8192, None) == -1
+    assert call(t=65540) == -3 and call(pos=2050) == -3
+    assert lib.pec_rope_table_floats(0) == 8192 and lib.pec_rope_table_floats(64) == 8192 + 128
+    assert lib.pec_rope_table_floats(65) == 8192 + 256 and lib.pec_rope_table_floats(-1) == 0
+    assert lib.pec_rope_table(500000.0, 10, 64, 4096, None) == -2
+    assert lib.pec_rope_table(0.0, 10, 128, 4096, None) == -1 and lib.pec_rope_table(1e4, 10, 128, None, None) == -1
+    assert lib.pec_rope_table(1e4, 10, 128, 4100, None) == -3
 
 
 def test_linear_merged_validates_on_the_host():
