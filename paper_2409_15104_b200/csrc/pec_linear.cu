@@ -9,7 +9,8 @@
 // operation of a single-CTA 128 x 256 tile - and keeps its 128 rows of the fp32 accumulator in its
 // own tensor memory (256 columns).  The even-ranked CTA (the leader) issues every tcgen05.mma; both
 // CTAs' loads count on the leader's "full" barrier and the leader's commits arrive on both CTAs'
-// barriers.  Warps 0-3 of each CTA read its accumulator rows back, round to bf16 and store.  Two
+// barriers.  Warps 0-3 of each CTA read its accumulator rows back, round to bf16, lay them out in the (by then free)
+// operand ring and hand them to the TMA in boxes of 32 rows x 64 columns.  Two
 // CTAs (of different pairs) fit on an SM (2 x 96 KB, 2 x 256 TMEM columns), so one's epilogue and
 // load latency hide under the other's MMAs.  Tensor-bound: 2 * M * N * K operations.
 #include <cuda.h>
@@ -18,6 +19,7 @@
 #include "pec_host.h"
 #include "pec_internal.h"
 #include "pec_sm100.cuh"
+#include "pec_tma_store.cuh"
 
 namespace pec {
 using namespace sm100;
@@ -62,35 +64,14 @@ struct Rope {
 };
 constexpr int kRopeFine = 64 * 64;
 
-// 32 accumulator columns -> bf16, 16 bytes per store, columns at or past N left out.
-__device__ __forceinline__ void store_chunk(__nv_bfloat16 *dst, const uint32_t (&r)[32], int col0, int32_t N)
+// 16 accumulator columns of row `lane` -> bf16 -> chunks `chunk`, `chunk` + 1 of a box (see pec_tma_store.cuh).
+__device__ __forceinline__ void box_put16(uint32_t box, int lane, int chunk, const uint32_t *r)
 {
 #pragma unroll
-    for (int i = 0; i < 32; i += 8) {
-        if (col0 + i < N) {
-            uint4 pk;
-            pk.x = pack_bf16(__uint_as_float(r[i + 0]), __uint_as_float(r[i + 1]));
-            pk.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-            pk.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-            pk.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
-            *reinterpret_cast<uint4 *>(dst + i) = pk;
-        }
-    }
-}
-
-__device__ __forceinline__ void store_chunk16(__nv_bfloat16 *dst, const uint32_t (&r)[16], int col0, int32_t N)
-{
-#pragma unroll
-    for (int i = 0; i < 16; i += 8) {
-        if (col0 + i < N) {
-            uint4 pk;
-            pk.x = pack_bf16(__uint_as_float(r[i + 0]), __uint_as_float(r[i + 1]));
-            pk.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-            pk.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-            pk.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
-            *reinterpret_cast<uint4 *>(dst + i) = pk;
-        }
-    }
+    for (int i = 0; i < 16; i += 8)
+        box_put(box, lane, chunk + (i >> 3),
+                pack_bf16(__uint_as_float(r[i + 0]), __uint_as_float(r[i + 1])), pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])),
+                pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5])), pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7])));
 }
 // Cosines and sines of sixteen channels i0 .. i0 + 15 for the row at position 64 a + b (see Rope).
 __device__ __forceinline__ void rope_angles(const float *table, int na, int a, int b, int i0, float (&c)[16], float (&s)[16])
@@ -124,8 +105,8 @@ __device__ __forceinline__ void tmem_ld16x2(uint32_t ta, uint32_t (&a)[16], uint
 
 template <bool kRope>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 2)
-linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-                   __nv_bfloat16 *y, int64_t y_stride, int64_t M, int32_t N, int32_t K, int32_t band, int32_t by_cols, int32_t *status,
+linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_y,
+              int64_t M, int32_t N, int32_t K, int32_t band, int32_t by_cols, int32_t *status,
               long long wait_cycles, int32_t test_skip_last_load, const Rope rope)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -167,7 +148,7 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
         for (int s = 0; s < kSlots; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
         mbar_init(smem_u32(&sh->acc_full), 1);
         mbar_init_fence();
-        prefetch_tmap(&tm_x); prefetch_tmap(&tm_w);
+        prefetch_tmap(&tm_x); prefetch_tmap(&tm_w); prefetch_tmap(&tm_y);
     }
     __syncthreads();
     // No early exit here: the two CTAs of a pair must take every collective step together (a CTA that
@@ -227,12 +208,23 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
         if (ok) {
             tc_fence_after();
             const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
+            // Every MMA has completed, so the operand ring is free: the warp's 32 rows x 256 columns leave through four
+            // boxes of 64 columns laid out there, each handed to the TMA as soon as it is complete.
+            const uint32_t boxes = ring + (uint32_t)warp * (4 * kStoreBoxBytes);
+            const int row0 = (int)m0 + warp * 32;
+            auto send = [&](int j) {                          // box j: columns n0 + 64 j .. + 63
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0 && row0 < M && n0 + 64 * j < N) box_store(&tm_y, boxes + j * kStoreBoxBytes, n0 + 64 * j, row0);
+            };
             if constexpr (!kRope) {
 #pragma unroll 1
                 for (int c = 0; c < kBN / 32; ++c) {
                     uint32_t r[32];
-                    tmem_ld32(taddr + c * 32, r);             // warp-wide; only the stores are predicated
-                    if (row < M) store_chunk(y + row * y_stride + n0 + c * 32, r, n0 + c * 32, N);
+                    tmem_ld32(taddr + c * 32, r);
+                    box_put16(boxes + (c >> 1) * kStoreBoxBytes, lane, (c & 1) * 4, r);
+                    box_put16(boxes + (c >> 1) * kStoreBoxBytes, lane, (c & 1) * 4 + 2, r + 16);
+                    if (c & 1) send(c >> 1);
                 }
             } else {
                 // The tile's 256 columns are two heads; a thread holds a whole row, so both channels of a pair are its own.
@@ -255,13 +247,15 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
                                 b[j] = __float_as_uint(xb * cf[j] + xa * sf[j]);
                             }
                         }
-                        if (row < M) {
-                            store_chunk16(y + row * y_stride + n0 + col_a, a, n0 + col_a, N);
-                            store_chunk16(y + row * y_stride + n0 + col_b, b, n0 + col_b, N);
-                        }
+                        box_put16(boxes + (2 * hh) * kStoreBoxBytes, lane, it * 2, a);         // columns 128 hh + 16 it ..
+                        box_put16(boxes + (2 * hh + 1) * kStoreBoxBytes, lane, it * 2, b);     // and their partners 64 on
                     }
                 }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) send(j);
             }
+            if (lane == 0) { bulk_commit(); bulk_wait_read(); }     // the boxes must outlive the TMA's reads of them
+            __syncwarp();
         }
     }
     tc_fence_before();
@@ -327,8 +321,9 @@ static int linear_common(const char *who, const void *x, int64_t x_stride, const
         }
     }
     if (M == 0) return PEC_OK;
-    CUtensorMap tm_x, tm_w;
-    if (!host::make_matrix_map(&tm_x, x, M, K, x_stride, lin::kBM) || !host::make_matrix_map(&tm_w, w, N, K, w_stride, 128)) {
+    CUtensorMap tm_x, tm_w, tm_y;
+    if (!host::make_matrix_map(&tm_x, x, M, K, x_stride, lin::kBM) || !host::make_matrix_map(&tm_w, w, N, K, w_stride, 128) ||
+        !host::make_matrix_map(&tm_y, y, M, N, y_stride, (int)sm100::kStoreBoxRows)) {
         set_error("%s: cuTensorMapEncodeTiled failed", who);
         return PEC_ERR_CUDA;
     }
@@ -357,12 +352,10 @@ static int linear_common(const char *who, const void *x, int64_t x_stride, const
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (rope)
         lin::linear_kernel<true><<<grid, lin::kThreads, lin::kSmemBytes, stream>>>(
-            tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, (int32_t)band, by_cols, status,
-            (long long)wait_limit_cycles(), test_skip_last_load(), *rope);
+            tm_x, tm_w, tm_y, M, N, K, (int32_t)band, by_cols, status, (long long)wait_limit_cycles(), test_skip_last_load(), *rope);
     else
         lin::linear_kernel<false><<<grid, lin::kThreads, lin::kSmemBytes, stream>>>(
-            tm_x, tm_w, static_cast<__nv_bfloat16 *>(y), y_stride, M, N, K, (int32_t)band, by_cols, status,
-            (long long)wait_limit_cycles(), test_skip_last_load(), lin::Rope{});
+            tm_x, tm_w, tm_y, M, N, K, (int32_t)band, by_cols, status, (long long)wait_limit_cycles(), test_skip_last_load(), lin::Rope{});
     const cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("%s: launch failed: %s", who, cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;
