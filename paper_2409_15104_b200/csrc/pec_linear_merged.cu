@@ -27,6 +27,7 @@
 #include "pec_host.h"
 #include "pec_internal.h"
 #include "pec_sm100.cuh"
+#include "pec_tma_store.cuh"
 
 namespace pec {
 using namespace sm100;
@@ -53,8 +54,7 @@ constexpr size_t kSmemBytes = kSlots * kSlotBytes + 1024 + sizeof(Shared);
 struct Params {
     const float *o[kMaxParts];
     const float *lse[kMaxParts];
-    __nv_bfloat16 *y;
-    int64_t y_stride, M;
+    int64_t M;
     int32_t N, Hq, band, by_cols, test_skip_last_load;
     int32_t *status;
     long long wait_cycles;
@@ -106,7 +106,7 @@ __device__ __forceinline__ bool wait_bar_cluster(uint32_t bar, uint32_t parity, 
 
 template <int kParts>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-linear_merged_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ Params p)
+linear_merged_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_y, const __grid_constant__ Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -146,7 +146,7 @@ linear_merged_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
         }
         mbar_init(smem_u32(&sh->acc_full), 1);
         mbar_init_fence();
-        prefetch_tmap(&tm_w);
+        prefetch_tmap(&tm_w); prefetch_tmap(&tm_y);
     }
     __syncthreads();
     cluster_sync();                                           // both CTAs' barriers exist before anyone signals them
@@ -277,33 +277,34 @@ linear_merged_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_cons
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(leader_addr(smem_u32(&sh->full[slot])));
         }
-        // Epilogue: warp w reads lane quarter w % 4 of column group w / 4 (128 columns), rounds to bf16 and stores.
+        // Epilogue: warp w reads lane quarter w % 4 of column group w / 4 (128 columns), rounds to bf16, lays its 32 rows
+        // out in the operand ring (free once every MMA has completed) as two boxes of 64 columns and hands them to the TMA.
         ok = __all_sync(0xffffffffu, ok && wait_bar(smem_u32(&sh->acc_full), 0, wctx));
         if (ok) {
             tc_fence_after();
             const int quarter = warp & 3, cgroup = warp >> 2;
-            const int64_t row = m0 + quarter * 32 + lane;
+            const int row0 = (int)m0 + quarter * 32;
             const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + cgroup * 128;
+            const uint32_t boxes = ring + (uint32_t)warp * (2 * kStoreBoxBytes);
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
                 uint32_t r[32];
-                tmem_ld32(taddr + c * 32, r);                 // warp-wide; only the stores are predicated
-                const int col0 = n0 + cgroup * 128 + c * 32;
-                if (row < p.M) {
-                    __nv_bfloat16 *dst = p.y + row * p.y_stride + col0;
+                tmem_ld32(taddr + c * 32, r);
+                const uint32_t box = boxes + (c >> 1) * kStoreBoxBytes;
 #pragma unroll
-                    for (int i = 0; i < 32; i += 8) {
-                        if (col0 + i < p.N) {
-                            uint4 pk;
-                            pk.x = pack_bf16(__uint_as_float(r[i + 0]), __uint_as_float(r[i + 1]));
-                            pk.y = pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-                            pk.z = pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-                            pk.w = pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
-                            *reinterpret_cast<uint4 *>(dst + i) = pk;
-                        }
-                    }
+                for (int i = 0; i < 32; i += 8)
+                    box_put(box, lane, (c & 1) * 4 + (i >> 3),
+                            pack_bf16(__uint_as_float(r[i + 0]), __uint_as_float(r[i + 1])), pack_bf16(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])),
+                            pack_bf16(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5])), pack_bf16(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7])));
+                if (c & 1) {
+                    const int col0 = n0 + cgroup * 128 + (c >> 1) * 64;
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && row0 < p.M && col0 < p.N) box_store(&tm_y, box, col0, row0);
                 }
             }
+            if (lane == 0) { bulk_commit(); bulk_wait_read(); }     // the boxes must outlive the TMA's reads of them
+            __syncwarp();
         }
     }
     tc_fence_before();
@@ -322,10 +323,10 @@ static bool prepare()
 }
 
 template <int kParts>
-static cudaError_t launch(dim3 grid, cudaStream_t stream, const CUtensorMap &tm_w, const Params &p)
+static cudaError_t launch(dim3 grid, cudaStream_t stream, const CUtensorMap &tm_w, const CUtensorMap &tm_y, const Params &p)
 {
     if (!prepare<kParts>()) return cudaErrorUnknown;
-    linear_merged_kernel<kParts><<<grid, kThreads, kSmemBytes, stream>>>(tm_w, p);
+    linear_merged_kernel<kParts><<<grid, kThreads, kSmemBytes, stream>>>(tm_w, tm_y, p);
     return cudaGetLastError();
 }
 
@@ -353,12 +354,14 @@ extern "C" int pec_linear_merged(const void *const *o_parts, const float *const 
     }
     if (!aligned) { set_error("pec_linear_merged: w, y and the parts must be 16-byte aligned, w and y with row strides that are multiples of 8"); return PEC_ERR_ALIGNMENT; }
     if (rows == 0) return PEC_OK;
-    CUtensorMap tm_w;
-    if (!host::make_matrix_map(&tm_w, w, N, K, w_stride, 128)) { set_error("pec_linear_merged: cuTensorMapEncodeTiled failed"); return PEC_ERR_CUDA; }
+    CUtensorMap tm_w, tm_y;
+    if (!host::make_matrix_map(&tm_w, w, N, K, w_stride, 128) || !host::make_matrix_map(&tm_y, y, rows, N, y_stride, (int)sm100::kStoreBoxRows)) {
+        set_error("pec_linear_merged: cuTensorMapEncodeTiled failed");
+        return PEC_ERR_CUDA;
+    }
     lmg::Params p = {};
     for (int i = 0; i < n; ++i) { p.o[i] = static_cast<const float *>(o_parts[i]); p.lse[i] = lse_parts[i]; }
-    p.y = static_cast<__nv_bfloat16 *>(y);
-    p.y_stride = y_stride; p.M = rows; p.N = N; p.Hq = Hq;
+    p.M = rows; p.N = N; p.Hq = Hq;
     p.status = status; p.wait_cycles = (long long)wait_limit_cycles(); p.test_skip_last_load = test_skip_last_load();
     const int64_t pairs = (rows + 2 * lmg::kBM - 1) / (2 * lmg::kBM), gn = (N + lmg::kBN - 1) / lmg::kBN;
     if (gn > 65535) { set_error("pec_linear_merged: N too large"); return PEC_ERR_UNSUPPORTED; }
@@ -378,14 +381,14 @@ extern "C" int pec_linear_merged(const void *const *o_parts, const float *const 
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     cudaError_t err = cudaErrorUnknown;
     switch (n) {
-    case 1: err = lmg::launch<1>(grid, stream, tm_w, p); break;
-    case 2: err = lmg::launch<2>(grid, stream, tm_w, p); break;
-    case 3: err = lmg::launch<3>(grid, stream, tm_w, p); break;
-    case 4: err = lmg::launch<4>(grid, stream, tm_w, p); break;
-    case 5: err = lmg::launch<5>(grid, stream, tm_w, p); break;
-    case 6: err = lmg::launch<6>(grid, stream, tm_w, p); break;
-    case 7: err = lmg::launch<7>(grid, stream, tm_w, p); break;
-    case 8: err = lmg::launch<8>(grid, stream, tm_w, p); break;
+    case 1: err = lmg::launch<1>(grid, stream, tm_w, tm_y, p); break;
+    case 2: err = lmg::launch<2>(grid, stream, tm_w, tm_y, p); break;
+    case 3: err = lmg::launch<3>(grid, stream, tm_w, tm_y, p); break;
+    case 4: err = lmg::launch<4>(grid, stream, tm_w, tm_y, p); break;
+    case 5: err = lmg::launch<5>(grid, stream, tm_w, tm_y, p); break;
+    case 6: err = lmg::launch<6>(grid, stream, tm_w, tm_y, p); break;
+    case 7: err = lmg::launch<7>(grid, stream, tm_w, tm_y, p); break;
+    case 8: err = lmg::launch<8>(grid, stream, tm_w, tm_y, p); break;
     }
     if (err != cudaSuccess) { set_error("pec_linear_merged: launch failed: %s", cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;
