@@ -297,6 +297,47 @@ def test_partitioned_step_can_be_captured_and_replayed(pec):
     compare(runner.out_o, runner.out_l, *want, 2e-2, 1e-3, "graph replay")
 
 
+def test_decode_and_gemm_calls_capture_into_a_graph(pec):
+    """A decode step (slice kernel + its dependent merge kernel), the QKV GEMM with rotary encoding and the Eq. 5 GEMM on
+    unmerged partials, captured into one CUDA graph: the replay gives the eager calls' bits."""
+    L, hq, hkv, T, d = 5000, 16, 2, 300, 256
+    q, k, v = workloads.normal_tensor(14000, 1, (hq, 128), torch.bfloat16).to(DEV), *_gpu(*_qkv(14001, L, hq, hkv, torch.bfloat16)[1:])
+    x = workloads.normal_tensor(14002, 1, (T, d), torch.bfloat16).to(DEV)
+    w_qkv = (workloads.normal_tensor(14003, 2, ((hq + 2 * hkv) * 128, d), torch.float32) / d ** 0.5).to(torch.bfloat16).to(DEV)
+    w_l = (workloads.normal_tensor(14004, 3, (d, hq * 128), torch.float32) / (hq * 128) ** 0.5).to(torch.bfloat16).to(DEV)
+    tables = pec.pec_rope_table(500000.0, T, DEV)
+    os_, ls_ = _random_partials(14005, T, hq, 2)
+    os_, ls_ = [torch.nan_to_num(o).to(DEV) for o in os_], [l.to(DEV) for l in ls_]
+    o = torch.empty((hq, 128), dtype=torch.float32, device=DEV); lse = torch.empty((hq,), dtype=torch.float32, device=DEV)
+    a = pec.decode_args(q, k, v, o, lse, 0, L)
+    ws = torch.empty(max(pec.pec_decode_workspace_size(a), 16), dtype=torch.uint8, device=DEV)
+    y1 = torch.empty((T, (hq + 2 * hkv) * 128), dtype=torch.bfloat16, device=DEV)
+    y2 = torch.empty((T, d), dtype=torch.bfloat16, device=DEV)
+
+    def calls(stream=None):
+        pec.pec_decode_attn(q, k, v, o=o, lse=lse, workspace=ws, stream=stream)
+        pec.pec_linear_rope(x, w_qkv, tables, (hq + hkv) * 128, y=y1, stream=stream)
+        pec.pec_linear_merged(os_, ls_, w_l, y=y2, stream=stream)
+
+    calls()
+    torch.cuda.synchronize()
+    pec.check_status()
+    eager = [t.clone() for t in (o, lse, y1, y2)]
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            calls(stream)
+    for t in (o, lse, y1, y2):
+        t.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    pec.check_status()
+    for got, want in zip((o, lse, y1, y2), eager):
+        assert torch.equal(got, want)
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
 def test_non_causal_partition_of_a_chunk(pec, dtype):
     S, P, c0, n = 900, 3, 256, 300
