@@ -3,16 +3,20 @@
 // [T, (Hq + 2 Hkv) * 128] tensor whose slices pec_prefill_attn reads through strides) and the
 // post-self-attention linear layer (Eq. 5).
 //
-// A cluster of two CTAs computes one 256 x 256 tile of y with 256-row MMAs (cta_group::2).  Per K
-// step of 64 each CTA loads, by TMA into a 3-slot ring (128-byte swizzle, both operands K-major),
+// A cluster of two CTAs computes 256 x 256 tiles of y with 256-row MMAs (cta_group::2).  Per K
+// step of 64 each CTA loads, by TMA into a 6-slot ring (128-byte swizzle, both operands K-major),
 // its own 128 rows of x and 128 of the 256 rows of w - half the shared-memory operand traffic per
 // operation of a single-CTA 128 x 256 tile - and keeps its 128 rows of the fp32 accumulator in its
-// own tensor memory (256 columns).  The even-ranked CTA (the leader) issues every tcgen05.mma; both
-// CTAs' loads count on the leader's "full" barrier and the leader's commits arrive on both CTAs'
-// barriers.  Warps 0-3 of each CTA read its accumulator rows back, round to bf16, lay them out in the (by then free)
-// operand ring and hand them to the TMA in boxes of 32 rows x 64 columns.  Two
-// CTAs (of different pairs) fit on an SM (2 x 96 KB, 2 x 256 TMEM columns), so one's epilogue and
-// load latency hide under the other's MMAs.  Tensor-bound: 2 * M * N * K operations.
+// own tensor memory.  The even-ranked CTA (the leader) issues every tcgen05.mma; both CTAs' loads
+// count on the leader's "full" barrier and the leader's commits arrive on both CTAs' barriers.
+// The kernel is persistent: one pair per two SMs walks every (number of pairs)-th tile of a banded
+// tile order, the operand ring runs on through the tile boundaries and the accumulator is double-
+// buffered (2 x 256 tensor-memory columns), so the MMAs of the next tile run while warps 0-3 of each
+// CTA read the finished one out (a lane = a row), round to bf16, lay their rows out in staging
+// boxes of 32 rows x 64 columns and hand those to the TMA; the pair's barriers, tensor memory and
+// first loads' latency are paid once per CTA, not per tile.  "Accumulator free" is signalled to
+// the leader by all eight reading warps of the pair (cluster-scope release / acquire).
+// Tensor-bound: 2 * M * N * K operations.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -26,20 +30,11 @@ using namespace sm100;
 
 namespace lin {
 constexpr int kBM = 128, kBN = 256, kBK = 64;
-constexpr int kSlots = 3;                                   // 96 KB per CTA: two CTAs share an SM
+constexpr int kSlots = 6;                                   // 192 KB of operands in flight per CTA
 constexpr int kThreads = 192;                               // 4 epilogue warps, MMA warp, loader warp
 constexpr uint32_t kABytes = kBM * kBK * 2;                 // this CTA's 128 rows of x
 constexpr uint32_t kWBytes = 128 * kBK * 2;                 // this CTA's half of the 256 rows of w
 constexpr uint32_t kSlotBytes = kABytes + kWBytes;          // 32 KB
-constexpr uint32_t kTmemCols = 256;
-
-struct Shared {
-    uint64_t full[kSlots], empty[kSlots], acc_full;
-    uint32_t tmem_base;
-    volatile int abort_flag;
-};
-constexpr size_t kSmemBytes = kSlots * kSlotBytes + 1024 + sizeof(Shared);
-
 // What the waits of a CTA need: its abort flag, the caller's status word and the wait limit.
 struct WaitCtx { volatile int *abort_flag; int32_t *status; long long limit; };
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const WaitCtx &w)
@@ -103,59 +98,87 @@ __device__ __forceinline__ void tmem_ld16x2(uint32_t ta, uint32_t (&a)[16], uint
         : "r"(ta), "r"(tb) : "memory");
 }
 
+// ---------------------------------------------------------------------------------------------
+// The kernel: one CTA pair per two SMs walks its share of the tiles (see the head of the file).
+constexpr uint32_t kStageBytes = 4 * 2 * kStoreBoxBytes;    // four warps, two boxes each
+struct Shared {
+    uint64_t full[kSlots], empty[kSlots], acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+constexpr size_t kSmemBytes = kSlots * kSlotBytes + kStageBytes + 1024 + sizeof(Shared);
+
+__device__ __forceinline__ void arrive_cluster(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ bool wait_cluster(uint32_t bar, uint32_t parity, const WaitCtx &w)
+{
+    const long long t0 = clock64();
+    for (;;) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bar), "r"(parity), "r"(2000u) : "memory");
+        if (ok) return true;
+        if (*w.abort_flag) return false;
+        if (clock64() - t0 > w.limit) {
+            *w.abort_flag = 1;
+            if (w.status) atomicExch(w.status, (int)PEC_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+
+struct Tiles { int32_t pairs, gn, band, by_cols, n_clusters; int64_t total; };
+__device__ __forceinline__ void tile_of(const Tiles &t, int64_t seq, int &pair_i, int &col_i)
+{
+    if (!t.by_cols) {
+        const int band_i = (int)(seq / ((int64_t)t.band * t.gn));
+        const int band_pairs = (t.pairs - band_i * t.band) < t.band ? (t.pairs - band_i * t.band) : t.band;
+        const int within = (int)(seq - (int64_t)band_i * t.band * t.gn);
+        pair_i = band_i * t.band + within % band_pairs;
+        col_i = within / band_pairs;
+    } else {
+        const int band_i = (int)(seq / ((int64_t)t.band * t.pairs));
+        const int band_cols = (t.gn - band_i * t.band) < t.band ? (t.gn - band_i * t.band) : t.band;
+        const int within = (int)(seq - (int64_t)band_i * t.band * t.pairs);
+        col_i = band_i * t.band + within % band_cols;
+        pair_i = within / band_cols;
+    }
+}
+
 template <bool kRope>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 2)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_y,
-              int64_t M, int32_t N, int32_t K, int32_t band, int32_t by_cols, int32_t *status,
-              long long wait_cycles, int32_t test_skip_last_load, const Rope rope)
+                         int64_t M, int32_t N, int32_t K, const Tiles tiles, int32_t *status,
+                         long long wait_cycles, int32_t test_skip_last_load, const Rope rope)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;
-    Shared *sh = reinterpret_cast<Shared *>(smem_raw + (ring - raw) + kSlots * kSlotBytes);
+    const uint32_t stage = ring + kSlots * kSlotBytes;
+    Shared *sh = reinterpret_cast<Shared *>(smem_raw + (ring - raw) + kSlots * kSlotBytes + kStageBytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_ctarank();                  // 0 = leader
-    // Tile order.  Clusters are dispatched x-fastest; taken as they come (all row pairs of one column
-    // of y, then the next column) every column would stream the whole of x from HBM again.  The
-    // dispatch index is re-read in bands.  by_cols == 0: bands of `band` row pairs, within a band the row
-    // pairs vary fastest and the columns next, so a band's rows of x stay in L2 while its columns are done
-    // (x is read once, w once per band).  by_cols == 1: bands of `band` columns of y, within a band the
-    // columns vary fastest and the row pairs next (w is read once, x once per band).  The host picks the
-    // cheaper of the two.
-    const int pairs = (int)(gridDim.x >> 1), gn = (int)gridDim.y;
-    const int64_t seq = (int64_t)blockIdx.y * pairs + (blockIdx.x >> 1);
-    int pair_i, col_i;
-    if (!by_cols) {
-        const int band_i = (int)(seq / ((int64_t)band * gn));
-        const int band_pairs = (pairs - band_i * band) < band ? (pairs - band_i * band) : band;
-        const int within = (int)(seq - (int64_t)band_i * band * gn);
-        pair_i = band_i * band + within % band_pairs;
-        col_i = within / band_pairs;
-    } else {
-        const int band_i = (int)(seq / ((int64_t)band * pairs));
-        const int band_cols = (gn - band_i * band) < band ? (gn - band_i * band) : band;
-        const int within = (int)(seq - (int64_t)band_i * band * pairs);
-        col_i = band_i * band + within % band_cols;
-        pair_i = within / band_cols;
-    }
-    const int64_t m0 = (int64_t)pair_i * (2 * kBM) + rank * kBM;
-    const int n0 = col_i * kBN;
+    const int cid = (int)(blockIdx.x >> 1);
     const int n_kb = (K + kBK - 1) / kBK;
     const WaitCtx wctx = {&sh->abort_flag, status, wait_cycles};
 
     if (tid == 0) {
         sh->abort_flag = (status && *reinterpret_cast<volatile int32_t *>(status) != 0) ? 1 : 0;
         for (int s = 0; s < kSlots; ++s) { mbar_init(smem_u32(&sh->full[s]), 1); mbar_init(smem_u32(&sh->empty[s]), 1); }
-        mbar_init(smem_u32(&sh->acc_full), 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&sh->acc_full[b]), 1); mbar_init(smem_u32(&sh->acc_empty[b]), 8); }
         mbar_init_fence();
         prefetch_tmap(&tm_x); prefetch_tmap(&tm_w); prefetch_tmap(&tm_y);
     }
     __syncthreads();
-    // No early exit here: the two CTAs of a pair must take every collective step together (a CTA that
-    // starts with the abort flag set simply lets its waits fail at once).
     cluster_sync();                                           // both CTAs' barriers exist before anyone signals them
     if (warp == 0) {
-        tmem_alloc_pair(smem_u32(&sh->tmem_base), kTmemCols);
+        tmem_alloc_pair(smem_u32(&sh->tmem_base), 512);
         tmem_relinquish_pair();
     }
     tc_fence_before();
@@ -165,15 +188,23 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
 
     if (warp == 5) {
         if (lane == 0) {
-            for (int kb = 0; kb < n_kb; ++kb) {
-                const int slot = kb % kSlots, fill = kb / kSlots;
-                if (test_skip_last_load && rank == 1 && kb == n_kb - 1) break;   // test hook: the pair's waits for this step run out
-                if (fill > 0 && !wait_bar(smem_u32(&sh->empty[slot]), (fill - 1) & 1, wctx)) break;
-                const uint32_t a = ring + slot * kSlotBytes;
-                const uint32_t bar = leader_addr(smem_u32(&sh->full[slot]));
-                if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[slot]), 2 * kSlotBytes);   // both CTAs' bytes
-                tma_load_2d_pair(a, &tm_x, bar, kb * kBK, (int)m0);
-                tma_load_2d_pair(a + kABytes, &tm_w, bar, kb * kBK, n0 + (int)rank * 128);
+            int it = 0;
+            bool ok = true;
+            for (int64_t seq = cid; seq < tiles.total && ok; seq += tiles.n_clusters) {
+                int pair_i, col_i;
+                tile_of(tiles, seq, pair_i, col_i);
+                const int m0 = pair_i * (2 * kBM) + (int)rank * kBM, n0 = col_i * kBN;
+                const bool last_tile = seq + tiles.n_clusters >= tiles.total;
+                for (int kb = 0; kb < n_kb; ++kb, ++it) {
+                    const int slot = it % kSlots, fill = it / kSlots;
+                    if (test_skip_last_load && rank == 1 && last_tile && kb == n_kb - 1) { ok = false; break; }   // test hook
+                    if (fill > 0 && !wait_bar(smem_u32(&sh->empty[slot]), (fill - 1) & 1, wctx)) { ok = false; break; }
+                    const uint32_t a = ring + slot * kSlotBytes;
+                    const uint32_t bar = leader_addr(smem_u32(&sh->full[slot]));
+                    if (rank == 0) mbar_arrive_expect_tx(smem_u32(&sh->full[slot]), 2 * kSlotBytes);   // both CTAs' bytes
+                    tma_load_2d_pair(a, &tm_x, bar, kb * kBK, m0);
+                    tma_load_2d_pair(a + kABytes, &tm_w, bar, kb * kBK, n0 + (int)rank * 128);
+                }
             }
         }
         __syncwarp();
@@ -181,89 +212,126 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc = idesc_bf16_f32(2 * kBM, kBN, 0, 0);
             bool ok = true;
-            for (int kb = 0; kb < n_kb && ok; ++kb) {
-                const int slot = kb % kSlots;
-                ok = wait_bar(smem_u32(&sh->full[slot]), (kb / kSlots) & 1, wctx);
-                if (!ok) break;
-                const uint32_t a = ring + slot * kSlotBytes, b = a + kABytes;
+            int it = 0, ti = 0;
+            for (int64_t seq = cid; seq < tiles.total && ok; seq += tiles.n_clusters, ++ti) {
+                const int b = ti & 1;
+                if (ti >= 2) {                                // both CTAs have read this accumulator's previous tile out
+                    ok = wait_cluster(smem_u32(&sh->acc_empty[b]), ((ti >> 1) - 1) & 1, wctx);
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                const uint32_t acc = tmem + b * 256;
+                for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
+                    const int slot = it % kSlots;
+                    ok = wait_bar(smem_u32(&sh->full[slot]), (it / kSlots) & 1, wctx);
+                    if (!ok) break;
+                    const uint32_t a = ring + slot * kSlotBytes, bb = a + kABytes;
 #pragma unroll
-                for (int ks = 0; ks < kBK / 16; ++ks)
-                    mma_ss_pair(tmem, smem_desc_sw128(a + ks * 32u, 16, 1024), smem_desc_sw128(b + ks * 32u, 16, 1024), idesc,
-                                (kb > 0 || ks > 0) ? 1u : 0u);
-                tc_commit_pair(smem_u32(&sh->empty[slot]));
+                    for (int ks = 0; ks < kBK / 16; ++ks)
+                        mma_ss_pair(acc, smem_desc_sw128(a + ks * 32u, 16, 1024), smem_desc_sw128(bb + ks * 32u, 16, 1024), idesc,
+                                    (kb > 0 || ks > 0) ? 1u : 0u);
+                    tc_commit_pair(smem_u32(&sh->empty[slot]));
+                }
+                if (ok) tc_commit_pair(smem_u32(&sh->acc_full[b]));
             }
-            if (ok) tc_commit_pair(smem_u32(&sh->acc_full));
         }
         __syncwarp();
     } else {
-        const int64_t row = m0 + warp * 32 + lane;
-        [[maybe_unused]] int rope_a = 0, rope_b = 0, rope_na = 0;
-        if constexpr (kRope) {
-            int64_t pos = 0;
-            if (row < M) pos = rope.positions ? (int64_t)rope.positions[row] : rope.pos0 + row;
-            pos = pos < 0 ? 0 : (pos >= rope.n_pos ? rope.n_pos - 1 : pos);
-            rope_a = (int)(pos >> 6); rope_b = (int)(pos & 63); rope_na = (rope.n_pos + 63) >> 6;
-        }
-        const bool ok = __all_sync(0xffffffffu, n_kb == 0 || wait_bar(smem_u32(&sh->acc_full), 0, wctx));
-        if (ok) {
+        const uint32_t boxes = stage + (uint32_t)warp * (2 * kStoreBoxBytes);
+        int ti = 0, n_sent = 0;
+        bool ok = true;
+        for (int64_t seq = cid; seq < tiles.total && ok; seq += tiles.n_clusters, ++ti) {
+            int pair_i, col_i;
+            tile_of(tiles, seq, pair_i, col_i);
+            const int m0 = pair_i * (2 * kBM) + (int)rank * kBM, n0 = col_i * kBN;
+            const int b = ti & 1;
+            const int row0 = m0 + warp * 32;
+            const int64_t row = (int64_t)row0 + lane;
+            [[maybe_unused]] int rope_a = 0, rope_b = 0, rope_na = 0;
+            if constexpr (kRope) {
+                int64_t pos = 0;
+                if (row < M) pos = rope.positions ? (int64_t)rope.positions[row] : rope.pos0 + row;
+                pos = pos < 0 ? 0 : (pos >= rope.n_pos ? rope.n_pos - 1 : pos);
+                rope_a = (int)(pos >> 6); rope_b = (int)(pos & 63); rope_na = (rope.n_pos + 63) >> 6;
+            }
+            ok = __all_sync(0xffffffffu, wait_bar(smem_u32(&sh->acc_full[b]), (ti >> 1) & 1, wctx));
+            if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16);
-            // Every MMA has completed, so the operand ring is free: the warp's 32 rows x 256 columns leave through four
-            // boxes of 64 columns laid out there, each handed to the TMA as soon as it is complete.
-            const uint32_t boxes = ring + (uint32_t)warp * (4 * kStoreBoxBytes);
-            const int row0 = (int)m0 + warp * 32;
-            auto send = [&](int j) {                          // box j: columns n0 + 64 j .. + 63
+            const uint32_t taddr = tmem + ((uint32_t)(warp * 32) << 16) + b * 256;
+            // A staging box may be written again once the TMA has read what was sent from it two boxes ago.
+            auto box_for = [&]() {
+                if (n_sent >= 2) { if (lane == 0) bulk_wait_read_1(); __syncwarp(); }
+                return boxes + (uint32_t)(n_sent & 1) * kStoreBoxBytes;
+            };
+            auto send = [&](uint32_t box, int j) {            // columns n0 + 64 j .. + 63
                 fence_async_smem();
                 __syncwarp();
-                if (lane == 0 && row0 < M && n0 + 64 * j < N) box_store(&tm_y, boxes + j * kStoreBoxBytes, n0 + 64 * j, row0);
+                if (lane == 0) {
+                    if (row0 < M && n0 + 64 * j < N) box_store(&tm_y, box, n0 + 64 * j, row0);
+                    bulk_commit();
+                }
+                ++n_sent;
             };
             if constexpr (!kRope) {
 #pragma unroll 1
-                for (int c = 0; c < kBN / 32; ++c) {
+                for (int j = 0; j < 4; ++j) {
                     uint32_t r[32];
-                    tmem_ld32(taddr + c * 32, r);
-                    box_put16(boxes + (c >> 1) * kStoreBoxBytes, lane, (c & 1) * 4, r);
-                    box_put16(boxes + (c >> 1) * kStoreBoxBytes, lane, (c & 1) * 4 + 2, r + 16);
-                    if (c & 1) send(c >> 1);
+                    const uint32_t box = box_for();
+                    tmem_ld32(taddr + j * 64, r);
+                    box_put16(box, lane, 0, r);
+                    box_put16(box, lane, 2, r + 16);
+                    tmem_ld32(taddr + j * 64 + 32, r);
+                    box_put16(box, lane, 4, r);
+                    box_put16(box, lane, 6, r + 16);
+                    if (j == 3) {                             // the accumulator is in registers / shared memory: hand it back
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) arrive_cluster(leader_addr(smem_u32(&sh->acc_empty[b])));
+                    }
+                    send(box, j);
                 }
             } else {
-                // The tile's 256 columns are two heads; a thread holds a whole row, so both channels of a pair are its own.
-                // Sixteen pairs of both heads per step, so a row's cosines and sines are worked out once per tile.
-                const bool turn0 = n0 < rope.rot_cols, turn1 = n0 + 128 < rope.rot_cols;    // rot_cols: whole heads
+                // Two heads per tile; per head two boxes (channels 0-63 and their partners 64-127), sixteen pairs per step.
+                const bool turn[2] = {n0 < rope.rot_cols, n0 + 128 < rope.rot_cols};
 #pragma unroll 1
-                for (int it = 0; it < 4; ++it) {              // channels 16 it .. 16 it + 15 and their partners, both heads
-                    float cf[16], sf[16];
-                    if (turn0) rope_angles(rope.table, rope_na, rope_a, rope_b, it * 16, cf, sf);   // a tile of value heads needs none
-#pragma unroll
-                    for (int hh = 0; hh < 2; ++hh) {
-                        const int col_a = hh * 128 + it * 16, col_b = col_a + 64;
-                        uint32_t a[16], b[16];
-                        tmem_ld16x2(taddr + col_a, a, taddr + col_b, b);
-                        if (hh == 0 ? turn0 : turn1) {
+                for (int hh = 0; hh < 2; ++hh) {
+                    if (n_sent > 0) { if (lane == 0) bulk_wait_read(); __syncwarp(); }   // both boxes are written side by side
+                    const uint32_t box_a = boxes, box_b = boxes + kStoreBoxBytes;
+#pragma unroll 1
+                    for (int it = 0; it < 4; ++it) {
+                        float cf[16], sf[16];
+                        if (turn[hh]) rope_angles(rope.table, rope_na, rope_a, rope_b, it * 16, cf, sf);
+                        uint32_t a[16], bq[16];
+                        tmem_ld16x2(taddr + hh * 128 + it * 16, a, taddr + hh * 128 + 64 + it * 16, bq);
+                        if (turn[hh]) {
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
-                                const float xa = __uint_as_float(a[j]), xb = __uint_as_float(b[j]);
+                                const float xa = __uint_as_float(a[j]), xb = __uint_as_float(bq[j]);
                                 a[j] = __float_as_uint(xa * cf[j] - xb * sf[j]);
-                                b[j] = __float_as_uint(xb * cf[j] + xa * sf[j]);
+                                bq[j] = __float_as_uint(xb * cf[j] + xa * sf[j]);
                             }
                         }
-                        box_put16(boxes + (2 * hh) * kStoreBoxBytes, lane, it * 2, a);         // columns 128 hh + 16 it ..
-                        box_put16(boxes + (2 * hh + 1) * kStoreBoxBytes, lane, it * 2, b);     // and their partners 64 on
+                        box_put16(box_a, lane, it * 2, a);
+                        box_put16(box_b, lane, it * 2, bq);
                     }
+                    if (hh == 1) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) arrive_cluster(leader_addr(smem_u32(&sh->acc_empty[b])));
+                    }
+                    send(box_a, 2 * hh);
+                    send(box_b, 2 * hh + 1);
                 }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) send(j);
             }
-            if (lane == 0) { bulk_commit(); bulk_wait_read(); }     // the boxes must outlive the TMA's reads of them
-            __syncwarp();
         }
+        if (lane == 0) bulk_wait_read();                      // the boxes must outlive the TMA's reads of them
+        __syncwarp();
     }
     tc_fence_before();
     __syncthreads();
     cluster_sync();                                           // the partner is done with this CTA's memory too
-    if (warp == 0) tmem_dealloc_pair(tmem, kTmemCols);
+    if (warp == 0) tmem_dealloc_pair(tmem, 512);
 }
-
 }  // namespace lin
 }  // namespace pec
 
@@ -328,34 +396,40 @@ static int linear_common(const char *who, const void *x, int64_t x_stride, const
         return PEC_ERR_CUDA;
     }
     static unsigned char ready[host::kMaxDevices] = {};
+    static int sm_count[host::kMaxDevices] = {};
     static std::mutex ready_mutex;
     if (!host::once_per_device(ready, ready_mutex, [] {
+            int dev = 0, sms = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+            sm_count[dev] = sms;
             return cudaFuncSetAttribute(lin::linear_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::kSmemBytes) == cudaSuccess &&
                    cudaFuncSetAttribute(lin::linear_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::kSmemBytes) == cudaSuccess; })) {
         set_error("%s: cannot raise the shared-memory limit: %s", who, cudaGetErrorString(cudaGetLastError()));
         return PEC_ERR_CUDA;
     }
+    int dev = 0;
+    cudaGetDevice(&dev);
     const int64_t pairs = (M + 2 * lin::kBM - 1) / (2 * lin::kBM), gn = (N + lin::kBN - 1) / lin::kBN;
-    if (gn > 65535) { set_error("%s: N too large", who); return PEC_ERR_UNSUPPORTED; }
-    // Bands of about 24 MB of one operand (4 to 32 tiles).  Measured on [32768, 4096] x [6144, 4096]^T with bands of
-    // row pairs: 12 (24 MB) 1409 TFLOP/s, 4: 1382, 8: 1404, 16: 1401, 23: 1385, 32: 1348 - the L2 serves both dies and
-    // also carries the other operand and the stream of y, so far less than its 126 MB holds a band.  Bands of x
-    // rows read x once and w once per band; bands of w rows (columns of y) the other way round: take the cheaper.
     const int64_t tile_bytes = (int64_t)2 * lin::kBM * K * 2;           // 256 rows of either operand
     int64_t band = ((int64_t)24 << 20) / tile_bytes;
     band = band < 4 ? 4 : (band > 32 ? 32 : band);
     const int64_t x_bytes = (int64_t)M * K * 2, w_bytes = (int64_t)N * K * 2;
     const int64_t by_rows_traffic = x_bytes + w_bytes * ((pairs + band - 1) / band);
     const int64_t by_cols_traffic = w_bytes + x_bytes * ((gn + band - 1) / band);
-    const int32_t by_cols = by_cols_traffic < by_rows_traffic ? 1 : 0;
-    dim3 grid((unsigned)(2 * pairs), (unsigned)gn);           // clusters of two CTAs along x
+    lin::Tiles tiles;
+    tiles.pairs = (int32_t)pairs; tiles.gn = (int32_t)gn; tiles.band = (int32_t)band;
+    tiles.by_cols = by_cols_traffic < by_rows_traffic ? 1 : 0;
+    tiles.total = pairs * gn;
+    const int64_t max_clusters = sm_count[dev] / 2 > 0 ? sm_count[dev] / 2 : 1;
+    tiles.n_clusters = (int32_t)(tiles.total < max_clusters ? tiles.total : max_clusters);
+    dim3 grid((unsigned)(2 * tiles.n_clusters));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (rope)
         lin::linear_kernel<true><<<grid, lin::kThreads, lin::kSmemBytes, stream>>>(
-            tm_x, tm_w, tm_y, M, N, K, (int32_t)band, by_cols, status, (long long)wait_limit_cycles(), test_skip_last_load(), *rope);
+            tm_x, tm_w, tm_y, M, N, K, tiles, status, (long long)wait_limit_cycles(), test_skip_last_load(), *rope);
     else
         lin::linear_kernel<false><<<grid, lin::kThreads, lin::kSmemBytes, stream>>>(
-            tm_x, tm_w, tm_y, M, N, K, (int32_t)band, by_cols, status, (long long)wait_limit_cycles(), test_skip_last_load(), lin::Rope{});
+            tm_x, tm_w, tm_y, M, N, K, tiles, status, (long long)wait_limit_cycles(), test_skip_last_load(), lin::Rope{});
     const cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("%s: launch failed: %s", who, cudaGetErrorString(err)); return PEC_ERR_CUDA; }
     return PEC_OK;
