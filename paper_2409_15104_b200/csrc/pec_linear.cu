@@ -30,7 +30,10 @@ using namespace sm100;
 
 namespace lin {
 constexpr int kBM = 128, kBN = 256, kBK = 64;
-constexpr int kSlots = 6;                                   // 192 KB of operands in flight per CTA
+constexpr int kMaxSlots = 6;
+// Operand ring and staging boxes per warp: 6 slots (192 KB) + 2 boxes; with the rotary encoding 5 slots + 4 boxes, so that
+// both heads of a tile are staged side by side and a row's cosines and sines are worked out once per tile.  224 KB either way.
+template <bool kRope> struct Cfg { static constexpr int kSlots = kRope ? 5 : 6, kBoxes = kRope ? 4 : 2; };
 constexpr int kThreads = 192;                               // 4 epilogue warps, MMA warp, loader warp
 constexpr uint32_t kABytes = kBM * kBK * 2;                 // this CTA's 128 rows of x
 constexpr uint32_t kWBytes = 128 * kBK * 2;                 // this CTA's half of the 256 rows of w
@@ -100,13 +103,12 @@ __device__ __forceinline__ void tmem_ld16x2(uint32_t ta, uint32_t (&a)[16], uint
 
 // ---------------------------------------------------------------------------------------------
 // The kernel: one CTA pair per two SMs walks its share of the tiles (see the head of the file).
-constexpr uint32_t kStageBytes = 4 * 2 * kStoreBoxBytes;    // four warps, two boxes each
 struct Shared {
-    uint64_t full[kSlots], empty[kSlots], acc_full[2], acc_empty[2];
+    uint64_t full[kMaxSlots], empty[kMaxSlots], acc_full[2], acc_empty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
 };
-constexpr size_t kSmemBytes = kSlots * kSlotBytes + kStageBytes + 1024 + sizeof(Shared);
+template <bool kRope> constexpr size_t smem_bytes() { return Cfg<kRope>::kSlots * kSlotBytes + 4 * Cfg<kRope>::kBoxes * kStoreBoxBytes + 1024 + sizeof(Shared); }
 
 __device__ __forceinline__ void arrive_cluster(uint32_t cluster_bar)
 {
@@ -160,8 +162,9 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;
+    constexpr int kSlots = Cfg<kRope>::kSlots, kBoxes = Cfg<kRope>::kBoxes;
     const uint32_t stage = ring + kSlots * kSlotBytes;
-    Shared *sh = reinterpret_cast<Shared *>(smem_raw + (ring - raw) + kSlots * kSlotBytes + kStageBytes);
+    Shared *sh = reinterpret_cast<Shared *>(smem_raw + (ring - raw) + kSlots * kSlotBytes + 4 * kBoxes * kStoreBoxBytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_ctarank();                  // 0 = leader
     const int cid = (int)(blockIdx.x >> 1);
@@ -237,7 +240,7 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
         }
         __syncwarp();
     } else {
-        const uint32_t boxes = stage + (uint32_t)warp * (2 * kStoreBoxBytes);
+        const uint32_t boxes = stage + (uint32_t)warp * (kBoxes * kStoreBoxBytes);
         int ti = 0, n_sent = 0;
         bool ok = true;
         for (int64_t seq = cid; seq < tiles.total && ok; seq += tiles.n_clusters, ++ti) {
@@ -291,19 +294,19 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
                     send(box, j);
                 }
             } else {
-                // Two heads per tile; per head two boxes (channels 0-63 and their partners 64-127), sixteen pairs per step.
-                const bool turn[2] = {n0 < rope.rot_cols, n0 + 128 < rope.rot_cols};
+                // Two heads per tile, two boxes per head (channels 0-63 and their partners 64-127), all four staged side by
+                // side; sixteen pairs of both heads per step, so a row's cosines and sines are worked out once per tile.
+                if (n_sent > 0) { if (lane == 0) bulk_wait_read(); __syncwarp(); }
+                const bool turn0 = n0 < rope.rot_cols, turn1 = n0 + 128 < rope.rot_cols;    // rot_cols: whole heads
 #pragma unroll 1
-                for (int hh = 0; hh < 2; ++hh) {
-                    if (n_sent > 0) { if (lane == 0) bulk_wait_read(); __syncwarp(); }   // both boxes are written side by side
-                    const uint32_t box_a = boxes, box_b = boxes + kStoreBoxBytes;
-#pragma unroll 1
-                    for (int it = 0; it < 4; ++it) {
-                        float cf[16], sf[16];
-                        if (turn[hh]) rope_angles(rope.table, rope_na, rope_a, rope_b, it * 16, cf, sf);
+                for (int it = 0; it < 4; ++it) {
+                    float cf[16], sf[16];
+                    if (turn0) rope_angles(rope.table, rope_na, rope_a, rope_b, it * 16, cf, sf);   // a tile of value heads needs none
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh) {
                         uint32_t a[16], bq[16];
                         tmem_ld16x2(taddr + hh * 128 + it * 16, a, taddr + hh * 128 + 64 + it * 16, bq);
-                        if (turn[hh]) {
+                        if (hh == 0 ? turn0 : turn1) {
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
                                 const float xa = __uint_as_float(a[j]), xb = __uint_as_float(bq[j]);
@@ -311,17 +314,15 @@ linear_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ 
                                 bq[j] = __float_as_uint(xb * cf[j] + xa * sf[j]);
                             }
                         }
-                        box_put16(box_a, lane, it * 2, a);
-                        box_put16(box_b, lane, it * 2, bq);
+                        box_put16(boxes + (2 * hh) * kStoreBoxBytes, lane, it * 2, a);
+                        box_put16(boxes + (2 * hh + 1) * kStoreBoxBytes, lane, it * 2, bq);
                     }
-                    if (hh == 1) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) arrive_cluster(leader_addr(smem_u32(&sh->acc_empty[b])));
-                    }
-                    send(box_a, 2 * hh);
-                    send(box_b, 2 * hh + 1);
                 }
+                tc_fence_before();                            // the accumulator is in shared memory: hand it back
+                __syncwarp();
+                if (lane == 0) arrive_cluster(leader_addr(smem_u32(&sh->acc_empty[b])));
+#pragma unroll
+                for (int j = 0; j < 4; ++j) send(boxes + j * kStoreBoxBytes, j);
             }
         }
         if (lane == 0) bulk_wait_read();                      // the boxes must outlive the TMA's reads of them
@@ -402,8 +403,8 @@ static int linear_common(const char *who, const void *x, int64_t x_stride, const
             int dev = 0, sms = 0;
             if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
             sm_count[dev] = sms;
-            return cudaFuncSetAttribute(lin::linear_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::kSmemBytes) == cudaSuccess &&
-                   cudaFuncSetAttribute(lin::linear_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::kSmemBytes) == cudaSuccess; })) {
+            return cudaFuncSetAttribute(lin::linear_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::smem_bytes<false>()) == cudaSuccess &&
+                   cudaFuncSetAttribute(lin::linear_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lin::smem_bytes<true>()) == cudaSuccess; })) {
         set_error("%s: cannot raise the shared-memory limit: %s", who, cudaGetErrorString(cudaGetLastError()));
         return PEC_ERR_CUDA;
     }
@@ -425,10 +426,10 @@ static int linear_common(const char *who, const void *x, int64_t x_stride, const
     dim3 grid((unsigned)(2 * tiles.n_clusters));
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (rope)
-        lin::linear_kernel<true><<<grid, lin::kThreads, lin::kSmemBytes, stream>>>(
+        lin::linear_kernel<true><<<grid, lin::kThreads, lin::smem_bytes<true>(), stream>>>(
             tm_x, tm_w, tm_y, M, N, K, tiles, status, (long long)wait_limit_cycles(), test_skip_last_load(), *rope);
     else
-        lin::linear_kernel<false><<<grid, lin::kThreads, lin::kSmemBytes, stream>>>(
+        lin::linear_kernel<false><<<grid, lin::kThreads, lin::smem_bytes<false>(), stream>>>(
             tm_x, tm_w, tm_y, M, N, K, tiles, status, (long long)wait_limit_cycles(), test_skip_last_load(), lin::Rope{});
     const cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) { set_error("%s: launch failed: %s", who, cudaGetErrorString(err)); return PEC_ERR_CUDA; }
