@@ -452,7 +452,8 @@ int pec_linear_merged(const void *const *o_parts, const float *const *lse_parts,
  *                               preemption works between kernels only) sets it lower.  value >= 1000.
  *   PEC_CTL_TEST_SKIP_LAST_LOAD test hook, 0 / 1: the loader of the tensor-core kernels leaves out its
  *                               last tile (attention: the last V tile of a CTA that walks at least two
- *                               key tiles; pec_linear, pec_linear_merged: the last K step of the second CTA of each pair),
+ *                               key tiles; pec_linear, pec_linear_merged: the last K step (pec_linear: of its last tile)
+ *                               of the second CTA of each pair),
  *                               so that the waits for it run out and the timeout path can be checked.
  *                               Results of such a launch are undefined; the status word tells.
  * Applies to launches enqueued after the call.  Errors: INVALID_ARG.
