@@ -213,7 +213,7 @@ def run_ours(args, wl):
         extra = {}
         for name, fn in (("c3", extra_partitioned), ("c3_merge_kernel", extra_merge_kernel), ("c4", run_preempted),
                          ("c2", run_short_batch), ("ring", run_ring), ("decode", run_decode), ("linear", run_linear),
-                         ("linear_merged", run_linear_merged)):
+                         ("linear_merged", run_linear_merged), ("layer", run_layer)):
             try:
                 extra[name] = fn(args)
             except Exception as exc:                       # an extra record must not take the headline with it
@@ -657,6 +657,63 @@ def run_linear_merged(args):
             "max_abs_err_vs_oracle_sampled_rows": err}
 
 
+def run_layer(args):
+    """Extra line: the attention part of one Llama-3-8B-shaped layer on a 32K-token request, every step through the
+    library - QKV generation with rotary encoding (Eq. 2), causal attention over 8 key partitions reading q, k, v as
+    strided slices of the fused tensor (Eq. 3-4), the post-attention linear layer (Eq. 5)."""
+    from paper_2409_15104_b200 import binding
+    from paper_2409_15104_b200.prefill import PartitionedPrefill
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    wl = workloads.WORKLOADS["c3"]
+    S, hq, hkv, d = wl.seq_len, wl.hq, wl.hkv, 4096
+    seed = workloads.BASE_SEED + 9
+    x = workloads.normal_tensor(seed, 1, (S, d), torch.bfloat16).to(dev)
+    w_qkv = (workloads.normal_tensor(seed, 2, ((hq + 2 * hkv) * 128, d), torch.float32) / d ** 0.5).to(torch.bfloat16).to(dev)
+    w_l = (workloads.normal_tensor(seed, 3, (d, hq * 128), torch.float32) / (hq * 128) ** 0.5).to(torch.bfloat16).to(dev)
+    tables = binding.pec_rope_table(500000.0, S, dev)
+    qkv = torch.empty((S, (hq + 2 * hkv) * 128), dtype=torch.bfloat16, device=dev)
+    y = torch.empty((S, d), dtype=torch.bfloat16, device=dev)
+    fused = qkv.view(S, hq + 2 * hkv, 128)
+    q, k, v = fused[:, :hq], fused[:, hq:hq + hkv], fused[:, hq + hkv:]
+    runner = PartitionedPrefill(S, hq, wl.num_parts, wl.dtype, dev, wl.part_align)
+
+    def step():
+        binding.pec_linear_rope(x, w_qkv, tables, (hq + hkv) * 128, y=qkv)
+        o, _ = runner.run(q, k, v)
+        binding.pec_linear(o.view(S, hq * 128), w_l, y=y)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    steps = _extra_steps(args, 20)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    binding.check_status()
+    ms = e0.elapsed_time(e1) / steps
+    flops = 2.0 * S * (hq + 2 * hkv) * 128 * d + workloads.attention_flops(workloads.causal_pairs(S), hq) + 2.0 * S * d * hq * 128
+    # the last rows of the layer's output against the oracle applied step by step to what each step actually read
+    import oracle
+    rows = [0, 1, 4095, S - 2, S - 1]
+    o_dev = runner.out_o
+    want_qkv = oracle.linear_rope(x[rows].cpu(), w_qkv.cpu(), rows, 500000.0, (hq + hkv) * 128)
+    err_qkv = float(np.abs(qkv[rows].float().cpu().double().numpy() - want_qkv).max())
+    want_o, _ = oracle.prefill_attn(q.cpu(), k.cpu(), v.cpu(), seq_len=S, rows=rows)
+    err_o = float(np.abs(o_dev[rows].float().cpu().double().numpy() - want_o).max())
+    want_y = oracle.linear(o_dev[rows].reshape(len(rows), hq * 128).cpu(), w_l.cpu())
+    err_y = float(np.abs(y[rows].float().cpu().double().numpy() - want_y).max())
+    return {"metric": "attention part of one layer (QKV generation + rotary encoding, attention, output projection), TFLOP/s (extra line)",
+            "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": ms, "steps": steps, "n_gpus": 1, "dtype": "bf16",
+            "data": "synthetic", "tokens_per_s": S / (ms * 1e-3),
+            "config": {"workload": f"layer: S={S}, model width {d}, {hq}/{hkv} heads, {wl.num_parts} key partitions",
+                       "l2": "activations exceed the L2"},
+            "max_abs_err_vs_oracle_sampled_rows": {"qkv": err_qkv, "o": err_o, "y": err_y}}
+
+
 def _short_batch(wl, dev, seed_offset=0):
     lens = workloads.short_lengths(wl.seed, wl.short_batch)
     cu = workloads.cu_seqlens(lens)
@@ -846,7 +903,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode", "linear", "linear_merged", "ring", "merge"], default="c5",
+    ap.add_argument("--workload", choices=["c2", "c3", "c4", "c5", "decode", "linear", "linear_merged", "layer", "ring", "merge"], default="c5",
                     help="c5 (default, the largest single-GPU configuration) and c3 print the full line; the others "
                          "print their extra record alone")
     ap.add_argument("--no-extra", action="store_true", help="skip the extra records nested under the headline line")
@@ -861,7 +918,7 @@ def main():
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU implementation")
-    alone = {"decode": run_decode, "linear": run_linear, "linear_merged": run_linear_merged, "ring": run_ring, "c2": run_short_batch, "c4": run_preempted,
+    alone = {"decode": run_decode, "linear": run_linear, "linear_merged": run_linear_merged, "layer": run_layer, "ring": run_ring, "c2": run_short_batch, "c4": run_preempted,
              "merge": extra_merge_kernel}
     if args.workload in alone:
         print(json.dumps(alone[args.workload](args)), flush=True)
