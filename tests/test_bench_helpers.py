@@ -30,3 +30,20 @@ def test_stored_counters_are_tied_to_the_kernel_sources():
     assert rec is not None and rec["captured_offline"] and rec["dram_bytes_per_launch"] > 0
     assert rec["stale"] == (rec["kernel_source_hash_at_capture"] != bench.kernel_source_hash())
     assert bench.stored_counters("no such workload") is None
+
+
+def test_gemm_roofline_takes_the_peak_that_matches_the_timed_region():
+    peaks = {"bf16_burst": 1600.0, "bf16_sustained": 1400.0, "hbm": 6500.0, "source": "measured"}
+    short = bench._gemm_roofline(1500.0, 40.0, peaks)                  # 40 ms timed: burst conditions
+    long = bench._gemm_roofline(1300.0, 5000.0, peaks)                 # 5 s timed: at the power cap
+    assert short["peak"] == 1600.0 and abs(short["frac"] - 1500.0 / 1600.0) < 1e-12
+    assert long["peak"] == 1400.0 and abs(long["frac"] - 1300.0 / 1400.0) < 1e-12
+    for r in (short, long):
+        assert abs(r["frac_of_burst"] - r["achieved"] / 1600.0) < 1e-12 and abs(r["frac_of_sustained"] - r["achieved"] / 1400.0) < 1e-12
+
+
+def test_the_stored_counters_of_the_headline_workload_are_current():
+    """roofline.traffic of the bench line comes from profiles/attn_counters.txt and is nulled when the attention kernel's
+    sources have changed since the capture: a change to those files must come with a new capture."""
+    for name in ("c3", "c5"):
+        assert not bench.stored_counters(name)["stale"], f"profiles/attn_counters.txt: the {name} capture is older than the kernel sources"
