@@ -207,3 +207,25 @@ def test_longest_paper_input_500k_ragged_eight_partitions_and_last_chunk(pec):
     want = oracle.prefill_attn(q, k, v, seq_len=S, rows=crow)
     idx = torch.as_tensor([r - c0 for r in crow], device=DEV)
     compare(oc[idx], lc[idx], *want, *TOL[torch.bfloat16], "S=500000 last chunk")
+
+
+def test_qkv_generation_at_full_size_on_sampled_rows(pec):
+    """The QKV GEMM of a 32K-token request (74 CTA pairs walking 42 tiles each), plain and with the rotary encoding:
+    rows next to every 256-row tile-pair boundary of the first and last bands plus seeded random rows, every column."""
+    M, K, N, theta = 32768, 4096, (32 + 2 * 8) * 128, 500000.0
+    x = workloads.normal_tensor(workloads.BASE_SEED + 7, 1, (M, K), torch.bfloat16)
+    w = (workloads.normal_tensor(workloads.BASE_SEED + 7, 2, (N, K), torch.float32) / K ** 0.5).to(torch.bfloat16)
+    dx, dw = x.to(DEV), w.to(DEV)
+    rows = sample_rows(M, [128, 256, 512, 3072, M - 512, M - 256, M - 128], 48, 707)
+    y = pec.pec_linear(dx, dw)
+    pec.check_status()
+    want = oracle.linear(x[rows], w)
+    err = float(np.abs(y[rows].float().cpu().double().numpy() - want).max())
+    tables = pec.pec_rope_table(theta, M, DEV)
+    y2 = pec.pec_linear_rope(dx, dw, tables, 40 * 128)
+    pec.check_status()
+    err2 = float(np.abs(y2[rows].float().cpu().double().numpy() - oracle.rope(want, rows, theta, 40 * 128)).max())
+    print(f"[parity] QKV GEMM 32768x6144x4096 on {len(rows)} rows: max|dy| = {err:.3e}, with rotary encoding {err2:.3e}")
+    assert err <= 2e-2 and err2 <= 2e-2
+    # the value heads are not turned: same bits as the plain GEMM there
+    assert torch.equal(y[:, 40 * 128:], y2[:, 40 * 128:])
