@@ -471,8 +471,29 @@ def extra_merge_kernel(args, name="c3"):
     byts = merge_bytes_exact(S, wl.hq, bounds, range(P), wl.dtype == torch.bfloat16)
     gbs = byts / (ms * 1e-3) / 1e9
     peaks = load_peaks()
+    # The two-way kernel (pec_attn_merge) on the same partials: the running merge of part 0's state with parts 1..P-1 in
+    # place, P - 1 launches; bytes per launch: state read, part read and state written for the part's live rows, the LSE alone for its empty rows.
+    acc_o, acc_l = o_parts[0].clone(), l_parts[0].clone()
+    def running():
+        for pp in range(1, P):
+            binding.pec_attn_merge(acc_o, acc_l, o_parts[pp], l_parts[pp], inplace=True)
+    running()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps2 = max(1, steps // 4)
+    e0.record()
+    for _ in range(reps2):
+        running()
+    e1.record()
+    torch.cuda.synchronize()
+    binding.check_status()
+    ms2 = e0.elapsed_time(e1) / (reps2 * (P - 1))
+    byts2 = sum(wl.hq * ((S - bounds[pp]) * 3 * 516 + bounds[pp] * 8) for pp in range(1, P)) / (P - 1)   # rows the part is empty for: the two LSEs
     return {"metric": "n-way LSE merge kernel, achieved HBM GB/s (extra record)", "value": gbs, "unit": "GB/s", "ms_per_launch": ms,
             "steps": steps, "parts": P,
+            "two_way_kernel": {"ms_per_launch": ms2, "gbs": byts2 / (ms2 * 1e-3) / 1e9, "frac": byts2 / (ms2 * 1e-3) / 1e9 / peaks["hbm"],
+                               "algorithmic_bytes_per_launch": byts2, "launches": reps2 * (P - 1),
+                               "what": "running in-place fp32 merge of the state with parts 1..P-1 (pec_attn_merge)"},
             "roofline": {"bound": "hbm", "kernel": "merge_n_kernel", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
                          "frac": gbs / peaks["hbm"], "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "traffic": None,
                          "algorithmic_bytes": byts, "peak_source": peaks["source"] + " copy bandwidth",

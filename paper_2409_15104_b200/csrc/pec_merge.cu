@@ -61,7 +61,7 @@ merge_kernel(const float *o_a, const float *lse_a, const float *__restrict__ o_b
                 b[u] = a[u];
                 if (i < n_here) {
                     const int64_t off = (base + i) * (kHeadDim / 4) + lane;
-                    if (fa[u] != 0.f) a[u] = ld_stream(reinterpret_cast<const float4 *>(o_a) + off);
+                    if (fa[u] != 0.f && !(kInplace && fb[u] == 0.f)) a[u] = ld_stream(reinterpret_cast<const float4 *>(o_a) + off);   // in place with an empty b: a stays, unread
                     if (fb[u] != 0.f) b[u] = ld_stream(reinterpret_cast<const float4 *>(o_b) + off);
                 }
             }
